@@ -1,0 +1,223 @@
+"""Pins of the CPU oracle's packing, binary dot, quantized product and recurrent steps."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1802_00150_b200 import synth
+
+
+def random_planes(k, n, seed, stream):
+    return np.where(synth.uniform01(k * n, seed, stream).reshape(k, n) < 0.5, -1, 1).astype(np.int8)
+
+
+# ---- packing ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n", [1, 31, 32, 33, 127, 128, 129, 300, 600])
+def test_pack_layout_and_roundtrip(n):
+    b = random_planes(1, n, 1, n)[0]
+    words = oracle.pack_plane(b)
+    assert words.size == 4 * ((n + 127) // 128) == oracle.words_per_row(n)
+    # bit j of word q is element 32q + j; pads are zero -- checked with numpy's own bit unpacking
+    bits = np.unpackbits(words.view(np.uint8), bitorder="little")
+    assert np.array_equal(bits[:n], (b > 0).astype(np.uint8))
+    assert not bits[n:].any()
+    assert np.array_equal(oracle.unpack_plane(words, n), b)
+
+
+# ---- XNOR / bitcount dot == the dot of the +-1 vectors (Appendix A) --------------------------------------
+
+def test_dot_xnor_equals_pm1_dot_all_lengths():
+    for n in range(1, 301):
+        a, b = random_planes(2, n, 2, n)
+        got = oracle.dot_xnor(oracle.pack_plane(a), oracle.pack_plane(b), n)
+        assert got == int(a.astype(np.int64) @ b.astype(np.int64))
+        assert got == oracle.dot_pm1(a, b)
+
+
+def test_dot_and_popc_identity():
+    # popc(a^b) = popc(a) + popc(b) - 2 popc(a&b)  =>  dot = n - 2popc(a) - 2popc(b) + 4popc(a&b)
+    for n in (17, 64, 200, 1000):
+        a, b = random_planes(2, n, 3, n)
+        pa, pb = oracle.pack_plane(a), oracle.pack_plane(b)
+        pc = lambda x: int(np.unpackbits(x.view(np.uint8)).sum())
+        assert oracle.dot_xnor(pa, pb, n) == n - 2 * pc(pa) - 2 * pc(pb) + 4 * pc(pa & pb)
+
+
+@pytest.mark.parametrize("n,lo,hi", [(300, 0, 300), (300, 0, 150), (300, 150, 300), (300, 31, 33), (300, 64, 64),
+                                     (257, 5, 250), (128, 32, 96)])
+def test_dot_xnor_range(n, lo, hi):
+    a, b = random_planes(2, n, 4, n + lo)
+    got = oracle.dot_xnor(oracle.pack_plane(a), oracle.pack_plane(b), n, lo, hi)
+    assert got == int(a[lo:hi].astype(np.int64) @ b[lo:hi].astype(np.int64))
+
+
+# ---- the quantized product (Sec. 4) ----------------------------------------------------------------------
+
+@pytest.mark.parametrize("m,n,kw,ka,batch", [(7, 50, 2, 2, 1), (33, 300, 3, 2, 3), (16, 129, 1, 4, 2), (5, 600, 4, 3, 2)])
+def test_product_equals_dense_product_of_reconstructions(m, n, kw, ka, batch):
+    W = synth.normal((m, n), 0.05, 5, 1).astype(np.float64)
+    X = synth.uniform((batch, n), -1, 1, 5, 2).astype(np.float64)
+    bias = synth.normal((m,), 0.1, 5, 3).astype(np.float64)
+    Wc, Wa = oracle.quantize_rows(W, kw, 2)
+    Xc, Xb = oracle.quantize_rows(X, ka, 2)
+    # reconstruct from the UNPACKED planes of an independent quantize call, row by row
+    What = np.stack([oracle.reconstruct(*oracle.quantize(W[r], kw, 2)) for r in range(m)])
+    Xhat = np.stack([oracle.reconstruct(*oracle.quantize(X[b], ka, 2)) for b in range(batch)])
+    y = oracle.binary_gemm(Wc, Wa, Xc, Xb, n, bias)
+    assert np.allclose(y, Xhat @ What.T + bias, rtol=1e-11, atol=1e-12)
+    # integer partials
+    D = oracle.binary_dots(Wc, Xc, n)
+    for bt in range(batch):
+        for r in (0, m - 1):
+            for i in range(kw):
+                for j in range(ka):
+                    wi = oracle.unpack_plane(Wc[r, i], n).astype(np.int64)
+                    xj = oracle.unpack_plane(Xc[bt, j], n).astype(np.int64)
+                    assert D[bt, r, i, j] == wi @ xj
+    # y from the partials, the formula of Fig. 3 (left)
+    y2 = np.einsum("ri,bj,brij->br", Wa, Xb, D.astype(np.float64)) + bias
+    assert np.allclose(y, y2, rtol=1e-12, atol=1e-13)
+
+
+def test_product_column_ranges_add_up():
+    m, n, I = 12, 200, 72
+    W = synth.normal((m, n), 0.05, 6, 1).astype(np.float64)
+    X = synth.normal((2, n), 1.0, 6, 2).astype(np.float64)
+    Wc, Wa = oracle.quantize_rows(W, 2, 2)
+    Xc, Xb = oracle.quantize_rows(X, 3, 2)
+    full = oracle.binary_gemm(Wc, Wa, Xc, Xb, n)
+    left = oracle.binary_gemm(Wc, Wa, Xc, Xb, n, lo=0, hi=I)
+    right = oracle.binary_gemm(Wc, Wa, Xc, Xb, n, lo=I, hi=n)
+    assert np.allclose(full, left + right, rtol=1e-12, atol=1e-13)
+
+
+# ---- recurrent steps -------------------------------------------------------------------------------------
+
+def dense_hat(codes, coeffs, n):
+    rows, k, _ = codes.shape
+    out = np.zeros((rows, n))
+    for r in range(rows):
+        for i in range(k):
+            out[r] += coeffs[r, i] * oracle.unpack_plane(codes[r, i], n)
+    return out
+
+
+def textbook_lstm(W, bias, x, h, c, H):
+    """Plain fp64 LSTM step (Eq. 6, gates i, f, o logistic and g tanh) on dense operands."""
+    p = np.concatenate([x, h], axis=1) @ W.T + (0 if bias is None else bias)
+    sig = lambda v: 1 / (1 + np.exp(-v))
+    i, f, o, g = sig(p[:, :H]), sig(p[:, H:2 * H]), sig(p[:, 2 * H:3 * H]), np.tanh(p[:, 3 * H:])
+    c2 = f * c + i * g
+    return o * np.tanh(c2), c2
+
+
+def textbook_gru(W, bias, x, h, I, H):
+    """Plain fp64 GRU step, linear-before-reset form, rows r, z, n; bias [b_r, b_z, b_nx, b_nh]."""
+    sig = lambda v: 1 / (1 + np.exp(-v))
+    px, ph = x @ W[:, :I].T, h @ W[:, I:].T
+    b = np.zeros(4 * H) if bias is None else bias
+    r = sig(px[:, :H] + ph[:, :H] + b[:H])
+    z = sig(px[:, H:2 * H] + ph[:, H:2 * H] + b[H:2 * H])
+    cand = np.tanh(px[:, 2 * H:] + b[2 * H:3 * H] + r * (ph[:, 2 * H:] + b[3 * H:]))
+    return (1 - z) * cand + z * h
+
+
+@pytest.mark.parametrize("I,H,batch,kw,ka", [(20, 12, 2, 2, 2), (33, 31, 1, 3, 3), (64, 40, 3, 2, 3)])
+def test_lstm_step_equals_textbook_step_on_reconstructed_operands(I, H, batch, kw, ka):
+    n = I + H
+    W = synth.normal((4 * H, n), 0.2, 7, 1).astype(np.float64)
+    bias = synth.normal((4 * H,), 0.1, 7, 2).astype(np.float64)
+    x = synth.normal((batch, I), 1.0, 7, 3).astype(np.float64)
+    h = synth.uniform((batch, H), -1, 1, 7, 4).astype(np.float64)
+    c = synth.uniform((batch, H), -1, 1, 7, 5).astype(np.float64)
+    Wc, Wa = oracle.quantize_rows(W, kw, 2)
+    zc, zb = oracle.quantize_rows(np.concatenate([x, h], axis=1), ka, 2)
+    What, zhat = dense_hat(Wc, Wa, n), dense_hat(zc, zb, n)
+    h_ref, c_ref = textbook_lstm(What, bias, zhat[:, :I], zhat[:, I:], c, H)
+    h_out, c_out = oracle.lstm_step(Wc, Wa, bias, I, H, x, h, c, ka, 2)
+    assert np.allclose(h_out, h_ref, rtol=1e-11, atol=1e-13) and np.allclose(c_out, c_ref, rtol=1e-11, atol=1e-13)
+    h_nb, _ = oracle.lstm_step(Wc, Wa, None, I, H, x, h, c, ka, 2)
+    assert np.allclose(h_nb, textbook_lstm(What, None, zhat[:, :I], zhat[:, I:], c, H)[0], rtol=1e-11, atol=1e-13)
+
+
+@pytest.mark.parametrize("I,H,batch,kw,ka", [(20, 12, 2, 2, 3), (32, 31, 1, 3, 3), (37, 40, 3, 2, 2)])
+def test_gru_step_equals_textbook_step_on_reconstructed_operands(I, H, batch, kw, ka):
+    n = I + H
+    W = synth.normal((3 * H, n), 0.2, 8, 1).astype(np.float64)
+    bias = synth.normal((4 * H,), 0.1, 8, 2).astype(np.float64)
+    x = synth.normal((batch, I), 1.0, 8, 3).astype(np.float64)
+    h = synth.uniform((batch, H), -1, 1, 8, 4).astype(np.float64)
+    Wc, Wa = oracle.quantize_rows(W, kw, 2)
+    zc, zb = oracle.quantize_rows(np.concatenate([x, h], axis=1), ka, 2)
+    What, zhat = dense_hat(Wc, Wa, n), dense_hat(zc, zb, n)
+    # the blend uses the UNQUANTIZED previous state h; the products use the quantized z
+    sig = lambda v: 1 / (1 + np.exp(-v))
+    px, ph = zhat[:, :I] @ What[:, :I].T, zhat[:, I:] @ What[:, I:].T
+    r = sig(px[:, :H] + ph[:, :H] + bias[:H])
+    z = sig(px[:, H:2 * H] + ph[:, H:2 * H] + bias[H:2 * H])
+    cand = np.tanh(px[:, 2 * H:] + bias[2 * H:3 * H] + r * (ph[:, 2 * H:] + bias[3 * H:]))
+    ref = (1 - z) * cand + z * h
+    got = oracle.gru_step(Wc, Wa, bias, I, H, x, h, ka, 2)
+    assert np.allclose(got, ref, rtol=1e-11, atol=1e-13)
+
+
+def exactly_representable(shape, a, c, seed, stream):
+    u = synth.uniform01(int(np.prod(shape)), seed, stream).reshape(shape)
+    return np.select([u < 0.25, u < 0.5, u < 0.75], [a + c, a - c, -a + c], -a - c)
+
+
+def test_cells_reduce_to_full_precision_cells_when_two_bits_are_exact():
+    # every weight row and the vector [x;h] take values in {+-a +-c}: 2-bit quantization is the identity,
+    # so the quantized step must equal the plain fp64 step on the unquantized operands
+    I, H, batch = 24, 16, 2
+    n = I + H
+    z = exactly_representable((batch, n), 0.5, 0.125, 9, 1)
+    x, h = z[:, :I], z[:, I:]
+    c = synth.uniform((batch, H), -1, 1, 9, 2).astype(np.float64)
+    Wl = exactly_representable((4 * H, n), 0.05, 0.02, 9, 3)
+    Wc, Wa = oracle.quantize_rows(Wl, 2, 2)
+    h_out, c_out = oracle.lstm_step(Wc, Wa, None, I, H, x, h, c, 2, 2)
+    h_ref, c_ref = textbook_lstm(Wl, None, x, h, c, H)
+    assert np.allclose(h_out, h_ref, atol=1e-12) and np.allclose(c_out, c_ref, atol=1e-12)
+    Wg = exactly_representable((3 * H, n), 0.05, 0.02, 9, 4)
+    Gc, Ga = oracle.quantize_rows(Wg, 2, 2)
+    got = oracle.gru_step(Gc, Ga, None, I, H, x, h, 2, 2)
+    assert np.allclose(got, textbook_gru(Wg, None, x, h, I, H), atol=1e-12)
+
+
+def test_sequences_are_repeated_steps():
+    I, H, batch, steps = 16, 8, 2, 4
+    W = synth.normal((4 * H, I + H), 0.3, 10, 1).astype(np.float64)
+    Wc, Wa = oracle.quantize_rows(W, 2, 2)
+    xs = synth.normal((steps, batch, I), 1.0, 10, 2).astype(np.float64)
+    h, c = np.zeros((batch, H)), np.zeros((batch, H))
+    h_seq, h_last, c_last = oracle.lstm_sequence(Wc, Wa, None, I, H, xs, h, c, 2, 2)
+    for s in range(steps):
+        h, c = oracle.lstm_step(Wc, Wa, None, I, H, xs[s], h, c, 2, 2)
+        assert np.array_equal(h_seq[s], h)
+    assert np.array_equal(h_last, h) and np.array_equal(c_last, c)
+    G = synth.normal((3 * H, I + H), 0.3, 10, 3).astype(np.float64)
+    Gc, Ga = oracle.quantize_rows(G, 2, 2)
+    h = np.zeros((batch, H))
+    g_seq, g_last = oracle.gru_sequence(Gc, Ga, None, I, H, xs, h, 3, 2)
+    for s in range(steps):
+        h = oracle.gru_step(Gc, Ga, None, I, H, xs[s], h, 3, 2)
+        assert np.array_equal(g_seq[s], h)
+    assert np.array_equal(g_last, h)
+
+
+def test_synth_is_reproducible_and_shaped():
+    a = synth.normal((4, 5), 0.03, 0, 1)
+    b = synth.normal((4, 5), 0.03, 0, 1)
+    assert a.dtype == np.float32 and np.array_equal(a, b)
+    assert not np.array_equal(a, synth.normal((4, 5), 0.03, 0, 2))
+    big = synth.normal((200000,), 1.0, 3, 1).astype(np.float64)
+    assert abs(big.mean()) < 0.01 and abs(big.std() - 1) < 0.01
+    u = synth.uniform((200000,), -1, 1, 3, 2).astype(np.float64)
+    assert abs(u.mean()) < 0.01 and abs(u.std() - 1 / np.sqrt(3)) < 0.01 and u.min() >= -1 and u.max() <= 1
+    # a prefix of a larger draw equals the smaller draw (counter-based)
+    assert np.array_equal(synth.uniform((10,), -1, 1, 5, 5), synth.uniform((20,), -1, 1, 5, 5)[:10])
+    wl = synth.WORKLOADS["lstm1024_b1"]
+    assert (wl.m, wl.n) == (4096, 2048)
+    ins = synth.inputs(wl)
+    assert ins["x_seq"].shape == (35, 1, 1024) and np.abs(ins["x_seq"]).max() <= 3.0

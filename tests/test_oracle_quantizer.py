@@ -1,0 +1,330 @@
+"""Pins of the CPU oracle's quantizer against what the paper and the mathematics fix.
+
+None of these re-types the oracle's own formula: each compares with a closed form the paper states,
+a library routine, brute force, or an invariant.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_1802_00150_b200 import synth
+
+
+def rows(kind, count, n, seed):
+    if kind == "normal":
+        return synth.normal((count, n), 1.0, seed, 11).astype(np.float64)
+    if kind == "uniform":
+        return synth.uniform((count, n), -1.0, 1.0, seed, 12).astype(np.float64)
+    if kind == "heavy":   # 90 % zeros-ish, 10 % large: alpha_1 < alpha_2 after the greedy step
+        u = synth.uniform01(count * n, seed, 13).reshape(count, n)
+        g = synth.normal((count, n), 1.0, seed, 14).astype(np.float64)
+        return np.where(u < 0.9, 0.01 * g, 10.0 + g)
+    raise ValueError(kind)
+
+
+# ---- k = 1: closed form alpha = mean|w|, b = sign(w)  (Sec. 2(c), Eq. 4) --------------------------------
+
+@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 600, 2048])
+@pytest.mark.parametrize("T", [0, 1, 2, 5])
+def test_k1_closed_form_and_fixed_point(n, T):
+    w = rows("normal", 1, n, 1)[0]
+    alpha, b = oracle.quantize(w, 1, T)
+    assert np.array_equal(b[0], np.where(w >= 0, 1, -1))
+    assert alpha[0] == pytest.approx(np.abs(w).mean(), rel=1e-14)
+
+
+def test_sign_of_zero_is_plus_one():
+    w = np.array([0.0, -0.0, 1.0, -1.0])
+    _, b = oracle.greedy(w, 1)
+    assert b[0].tolist() == [1, 1, 1, -1]
+
+
+# ---- greedy: each step is the optimal one-bit fit of the residue (Eq. 3-4) ------------------------------
+
+@pytest.mark.parametrize("kind", ["normal", "uniform", "heavy"])
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_greedy_invariants(kind, k):
+    w = rows(kind, 1, 777, 2)[0]
+    alpha, b = oracle.greedy(w, k)
+    assert np.all(alpha >= 0)
+    r = w.copy()
+    prev = np.linalg.norm(r)
+    for i in range(k):
+        assert alpha[i] == pytest.approx(np.abs(r).mean(), rel=1e-13, abs=1e-300)
+        assert np.array_equal(b[i], np.where(r >= 0, 1, -1))
+        # the one-bit optimum: no other scalar with these signs does better (closed form for a fixed b)
+        best_scalar = (b[i] * r).sum() / r.size
+        assert alpha[i] == pytest.approx(best_scalar, rel=1e-13, abs=1e-300)
+        r = r - alpha[i] * b[i]
+        assert np.linalg.norm(r) <= prev * (1 + 1e-15)
+        prev = np.linalg.norm(r)
+
+
+def test_greedy_heavy_tail_breaks_coefficient_order():
+    # alpha_1 >= alpha_2 is NOT an invariant of the greedy step: 90 % zeros + 10 % tens
+    w = np.array([0.0] * 90 + [10.0] * 10)
+    alpha, _ = oracle.greedy(w, 2)
+    assert alpha[0] == pytest.approx(1.0)
+    assert alpha[1] == pytest.approx(1.8)
+
+
+def test_greedy_uniform_limit():
+    # U(-1,1), n large: alpha_i -> 2^-i and relative MSE -> 4^-k (closed form of the recursion)
+    w = rows("uniform", 1, 400000, 3)[0]
+    for k in (1, 2, 3):
+        alpha, b = oracle.greedy(w, k)
+        assert np.allclose(alpha, [2.0 ** -(i + 1) for i in range(k)], atol=3e-3)
+        rel = oracle.objective(w, alpha, b) / (w ** 2).sum()
+        assert rel == pytest.approx(4.0 ** -k, rel=0.03)
+
+
+# ---- least-squares refit (Eq. 5) against a library solver -----------------------------------------------
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+@pytest.mark.parametrize("n", [5, 64, 1000])
+def test_ls_refit_matches_library_least_squares(k, n):
+    w = rows("normal", 1, n, 4)[0]
+    _, b = oracle.greedy(w, k)
+    alpha, solved = oracle.ls_refit(w, b)
+    B = b.T.astype(np.float64)
+    if np.linalg.matrix_rank(B) < k:
+        pytest.skip("rank-deficient draw")
+    assert solved
+    ref = np.linalg.lstsq(B, w, rcond=None)[0]          # SVD-based: independent of normal equations
+    assert np.allclose(alpha, ref, rtol=1e-10, atol=1e-12)
+    # residual orthogonal to every plane
+    assert np.abs(B.T @ (w - B @ alpha)).max() <= 1e-11 * np.abs(w).sum()
+
+
+def test_ls_refit_random_planes_not_from_greedy():
+    # planes unrelated to w, to catch a transposed or mis-indexed Gram matrix
+    n, k = 257, 3
+    w = rows("normal", 1, n, 5)[0]
+    b = np.where(synth.uniform01(k * n, 5, 20).reshape(k, n) < 0.5, -1, 1).astype(np.int8)
+    alpha, solved = oracle.ls_refit(w, b)
+    assert solved
+    assert np.allclose(alpha, np.linalg.lstsq(b.T.astype(float), w, rcond=None)[0], rtol=1e-10)
+
+
+def test_ls_refit_singular_is_skipped():
+    w = np.array([1.0, 2.0, 3.0, 4.0])
+    b = np.array([[1, 1, 1, 1], [1, 1, 1, 1]], dtype=np.int8)      # b_1 == b_2
+    alpha, solved = oracle.ls_refit(w, b, alpha_prev=[0.7, 0.1])
+    assert not solved and alpha.tolist() == [0.7, 0.1]
+    b[1] = -b[0]                                                    # b_1 == -b_2
+    _, solved = oracle.ls_refit(w, b, alpha_prev=[0.7, 0.1])
+    assert not solved
+
+
+# ---- level table and Algorithm 1 ------------------------------------------------------------------------
+
+def parse_fig1(golden_dir):
+    out = {}
+    for line in open(os.path.join(golden_dir, "fig1_two_bit.txt")):
+        if line.startswith("#") or ":" not in line:
+            continue
+        key, rest = line.split(":")
+        out[key.strip()] = [tuple(float(t) for t in part.split()) for part in rest.split("|")]
+    return out
+
+
+@pytest.mark.parametrize("a1,a2", [(1.0, 0.25), (0.8, 0.8), (2.0, 0.0), (0.5, 0.125)])
+def test_two_bit_levels_and_boundaries_as_fig1(golden_dir, a1, a2):
+    fig = parse_fig1(golden_dir)
+    v, code = oracle.levels([a1, a2])
+    assert np.allclose(v, [c1 * a1 + c2 * a2 for c1, c2 in fig["levels"]])
+    bounds = [c1 * a1 + c2 * a2 for c1, c2 in fig["boundaries"]]
+    # an entry just above a boundary takes the upper level, just below the lower one; the boundary goes up
+    eps = 1e-9
+    for p, t in enumerate(bounds):
+        if a2 == 0.0 or (a1 == a2 and p != 1):
+            continue                                   # duplicate levels: covered by the reconstruction test
+        for w, pos in ((t + eps, p + 1), (t - eps, p), (t, p + 1)):
+            b = oracle.bst(np.array([w]), [a1, a2])
+            assert oracle.reconstruct([a1, a2], b)[0] == pytest.approx(v[pos])
+
+
+@pytest.mark.parametrize("kind", ["normal", "uniform"])
+def test_two_bit_closed_form_codes(kind):
+    # Sec. 3: for alpha_1 >= alpha_2 >= 0, b_1 = sign(w), b_2 = sign(w - alpha_1 b_1)
+    w = rows(kind, 1, 5000, 6)[0]
+    for a1, a2 in [(1.0, 0.5), (0.9, 0.3), (0.6, 0.6 - 1e-9)]:
+        b = oracle.bst(w, [a1, a2])
+        b1 = np.where(w >= 0, 1, -1)
+        b2 = np.where(w - a1 * b1 >= 0, 1, -1)
+        assert np.array_equal(b[0], b1) and np.array_equal(b[1], b2)
+
+
+def nearest_level_ties_up(w, alpha):
+    k = len(alpha)
+    signs = np.array(list(itertools.product([-1.0, 1.0], repeat=k)))      # row c <-> code c, plane 1 = MSB
+    v = signs @ np.asarray(alpha, dtype=np.float64)
+    d = np.abs(w[:, None] - v[None, :])
+    best = d.min(axis=1)
+    # among the nearest levels take the largest value
+    cand = np.where(d <= best[:, None], v[None, :], -np.inf)
+    return cand.max(axis=1)
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_bst_is_nearest_level_for_any_real_coefficients(k):
+    w = rows("normal", 1, 3000, 7)[0]
+    draws = synth.normal((12, k), 1.0, 7, 30).astype(np.float64)          # negative / unsorted alphas too
+    for alpha in draws:
+        b = oracle.bst(w, alpha)
+        assert np.allclose(oracle.reconstruct(alpha, b), nearest_level_ties_up(w, alpha), rtol=0, atol=1e-12)
+
+
+def test_bst_duplicate_levels_reconstruction():
+    w = rows("normal", 1, 500, 8)[0]
+    for alpha in ([0.5, 0.5], [0.7, 0.0], [0.3, 0.3, 0.3], [0.0, 0.0]):
+        b = oracle.bst(w, alpha)
+        assert np.allclose(oracle.reconstruct(alpha, b), nearest_level_ties_up(w, np.array(alpha)), atol=1e-12)
+
+
+@pytest.mark.parametrize("k,n", [(1, 14), (2, 10), (2, 12), (3, 7), (4, 5)])
+def test_bst_codes_are_optimal_by_exhaustive_search(k, n):
+    # all (2^k)^n assignments of the whole vector, alpha fixed: the BST assignment attains the minimum
+    w = rows("normal", 1, n, 9 + k)[0]
+    alpha = np.abs(synth.normal((k,), 0.7, 9, 40).astype(np.float64)) + 0.05
+    b = oracle.bst(w, alpha)
+    got = oracle.objective(w, alpha, b)
+    signs = np.array(list(itertools.product([-1.0, 1.0], repeat=k)))
+    v = signs @ alpha                                                      # 2^k level values
+    m = 1 << k
+    head = min(n, 6)                                                       # enumerate the tail in chunks
+    tail = n - head
+    head_idx = np.array(list(itertools.product(range(m), repeat=head)))
+    head_err = ((w[None, :head] - v[head_idx]) ** 2).sum(axis=1)           # (m^head,)
+    best = np.inf
+    if tail == 0:
+        best = head_err.min()
+    else:
+        for tail_codes in itertools.product(range(m), repeat=tail):
+            e = ((w[head:] - v[list(tail_codes)]) ** 2).sum()
+            best = min(best, (head_err + e).min())
+    assert got <= best * (1 + 1e-12) + 1e-15
+    assert got >= best * (1 - 1e-12) - 1e-15
+
+
+# ---- Algorithm 2 ----------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kind", ["normal", "uniform", "heavy"])
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_alternating_objective_never_increases(kind, k):
+    for w in rows(kind, 6, 513, 20 + k):
+        T = 10
+        alpha, b, trace = oracle.quantize(w, k, T, with_trace=True)
+        assert trace.size == 1 + 2 * T
+        assert np.all(np.diff(trace) <= 1e-12 * trace[0])
+        # the trace's last entry is the objective of what is returned
+        assert trace[-1] == pytest.approx(oracle.objective(w, alpha, b), rel=1e-12, abs=1e-300)
+        ga, gb = oracle.greedy(w, k)
+        assert trace[0] == pytest.approx(oracle.objective(w, ga, gb), rel=1e-12)
+        assert trace[-1] <= trace[0] * (1 + 1e-12)
+
+
+def test_alternating_composition_matches_parts():
+    # Algorithm 2 is exactly: greedy, then T x (refit, BST) -- checked by driving the parts by hand
+    w = rows("normal", 1, 300, 31)[0]
+    for k, T in itertools.product((2, 3), (0, 1, 2, 3)):
+        alpha, b = oracle.greedy(w, k)
+        for _ in range(T):
+            alpha, _ = oracle.ls_refit(w, b, alpha_prev=alpha)
+            b = oracle.bst(w, alpha)
+        qa, qb = oracle.quantize(w, k, T)
+        assert np.array_equal(qa, alpha) and np.array_equal(qb, b)
+
+
+def test_method_ordering_on_synthetic_rows():
+    # error(alternating) <= error(refined greedy) <= error(greedy), the ordering of Tables 1-2, holds on
+    # Gaussian rows (the shape of trained weights).  Only alternating <= greedy is guaranteed in general
+    # (alternation starts from the greedy point); on heavy-tailed rows two cycles can lose to refined.
+    for kind in ("normal", "uniform", "heavy"):
+        worse = refined_worse = 0
+        for w in rows(kind, 8, 1024, 40):
+            for k in (2, 3, 4):
+                g = oracle.objective(w, *oracle.greedy(w, k))
+                r = oracle.objective(w, *oracle.refined_greedy(w, k))
+                a = oracle.objective(w, *oracle.quantize(w, k, 2))
+                assert a <= g * (1 + 1e-12)
+                refined_worse += r > g * (1 + 1e-9)
+                worse += a > r * (1 + 1e-9)
+        if kind == "normal":
+            assert worse == 0 and refined_worse == 0
+        if kind == "uniform":
+            assert worse <= 4 and refined_worse <= 6
+
+
+def gaussian_lloyd_max_mse(levels):
+    """MSE of the optimal `levels`-level scalar quantizer of N(0,1), by Lloyd iteration on the density."""
+    from scipy.stats import norm
+    q = np.linspace(-1.5, 1.5, levels)
+    for _ in range(500):
+        t = np.concatenate(([-np.inf], (q[:-1] + q[1:]) / 2, [np.inf]))
+        mass = norm.cdf(t[1:]) - norm.cdf(t[:-1])
+        q = (norm.pdf(t[:-1]) - norm.pdf(t[1:])) / mass
+    t = np.concatenate(([-np.inf], (q[:-1] + q[1:]) / 2, [np.inf]))
+    mass = norm.cdf(t[1:]) - norm.cdf(t[:-1])
+    return 1.0 - (q ** 2 * mass).sum()
+
+
+def test_gaussian_relative_mse_bracket():
+    w = rows("normal", 1, 200000, 50)[0]
+    e1 = oracle.objective(w, *oracle.quantize(w, 1, 2)) / (w ** 2).sum()
+    assert e1 == pytest.approx(1 - 2 / np.pi, rel=0.01)                   # one-bit optimum for a Gaussian
+    lm4 = gaussian_lloyd_max_mse(4)
+    assert lm4 == pytest.approx(0.1175, abs=5e-4)                         # textbook 4-level Lloyd-Max
+    greedy = oracle.objective(w, *oracle.greedy(w, 2)) / (w ** 2).sum()
+    prev = greedy
+    for T in (1, 2, 4, 8):
+        e = oracle.objective(w, *oracle.quantize(w, 2, T)) / (w ** 2).sum()
+        assert lm4 * (1 - 5e-3) <= e <= prev * (1 + 1e-12)
+        prev = e
+    # the 2-bit family {+-a1 +-a2} contains the symmetric 4-level optimum, so long runs approach it
+    assert prev <= lm4 * 1.02
+
+
+# ---- degenerate inputs ----------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_all_zero_vector(k):
+    alpha, b = oracle.quantize(np.zeros(37), k, 2)
+    assert np.all(alpha == 0) and np.all(b == 1)
+
+
+@pytest.mark.parametrize("k", [1, 2, 3])
+def test_constant_and_tiny_vectors_are_finite(k):
+    for w in (np.full(9, 0.3), np.array([-2.0]), np.array([1.0, -1.0]), np.array([5.0, 5.0, -5.0])):
+        alpha, b, trace = oracle.quantize(w, k, 3, with_trace=True)
+        assert np.all(np.isfinite(alpha)) and np.all(np.diff(trace) <= 1e-12)
+        assert np.allclose(oracle.reconstruct(alpha, b), w, atol=1e-12)   # these are exactly representable
+
+
+def test_exactly_representable_vector_is_reproduced():
+    # w in {+-a +-b}: two bits suffice, quantization is the identity after the refit
+    a, c = 0.75, 0.2
+    pattern = synth.uniform01(400, 60, 1)
+    w = np.select([pattern < 0.25, pattern < 0.5, pattern < 0.75], [a + c, a - c, -a + c], -a - c)
+    alpha, b = oracle.quantize(w, 2, 2)
+    assert np.allclose(oracle.reconstruct(alpha, b), w, atol=1e-13)
+    assert np.allclose(sorted(np.abs(alpha)), [c, a], atol=1e-13)
+
+
+# ---- the operation-count model --------------------------------------------------------------------------
+
+def test_cost_model_matches_the_paper(golden_dir):
+    for line in open(os.path.join(golden_dir, "cost_model.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        m, n, kw, kh, printed = line.split()
+        g = oracle.gamma(int(m), int(n), int(kw), int(kh))
+        assert g == pytest.approx(float(printed), rel=0.03)               # the paper says "roughly"
+    assert oracle.gamma(4096, 1024, 2, 2) == pytest.approx(7.67, abs=0.01)
+    assert oracle.gamma(4096, 1024, 3, 3) == pytest.approx(3.42, abs=0.01)
+    # quantizer: 2Tk^2 n binary + 2(T+1)kn non-binary; at T=2 the product model's 4k^2 n and 6kn terms
+    b, nb = oracle.quantizer_ops(1024, 3, 2)
+    assert b == 4 * 9 * 1024 and nb == 6 * 3 * 1024
