@@ -1,0 +1,416 @@
+"""Benchmark of the quantized recurrent hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path over one batch of synthetic input: for the recurrent
+workloads one full sequence (all timesteps: on-line quantization of [x;h], binary product, fused gate
+epilogue, every step), for the projection workload one bulk row-wise weight quantization plus one
+activation quantization and one binary product.  The headline value is LSTM/GRU timesteps per second
+(timesteps x concurrent sequences / time), summed over all GPUs; with N > 1 every rank runs its own
+independent sequences (weak scaling, no data-path collective).
+
+Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle on the host cores instead.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1802_00150_b200 import synth  # noqa: E402
+
+DEFAULT_WORKLOAD = "lstm1024_b1"
+METRIC = "quantized LSTM/GRU timesteps per second (timesteps x concurrent sequences / s)"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by workload; the summaries are under profiles/.  None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the cold-GEMV bandwidth line")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes_per_timestep(wl):
+    """What the method itself must move per timestep (all sequences of the batch): packed weight planes
+    once, the row coefficients, the fp32 activation [x;h] in, and the fp32 state in/out."""
+    words = (wl.n + 31) // 32
+    w_bytes = wl.k_w * wl.m * words * 4 + 4 * wl.k_w * wl.m
+    act = 4 * wl.n * wl.batch
+    state = (3 if wl.cell == "lstm" else 2) * 4 * wl.H * wl.batch
+    return w_bytes + act + state
+
+
+def units_per_step(wl):
+    return wl.steps * wl.batch if wl.cell != "proj" else 1
+
+
+# ---- reference arm: the CPU oracle, as it stands, on the host cores ------------------------------------
+
+def oracle_setup(wl, rows_limit=None):
+    import oracle
+    W = synth.weights(wl, rows=rows_limit).astype(np.float64)
+    Wc, Wa = oracle.quantize_rows(W, wl.k_w, wl.T)
+    return Wc, Wa
+
+
+def oracle_step(wl, Wc, Wa, ins, batch_limit=None):
+    """One benchmark step on the oracle; returns the number of units (timesteps x sequences) it covered."""
+    import oracle
+    if wl.cell == "proj":
+        acts = ins["acts"][:batch_limit].astype(np.float64)
+        Xc, Xb = oracle.quantize_rows(acts, wl.k_a, wl.T)
+        oracle.binary_gemm(Wc, Wa, Xc, Xb, wl.n)
+        return acts.shape[0] / wl.batch * (Wc.shape[0] / wl.m)
+    b = wl.batch if batch_limit is None else min(batch_limit, wl.batch)
+    xs, h0, c0 = ins["x_seq"][:, :b], ins["h0"][:b], ins["c0"][:b]
+    if wl.cell == "lstm":
+        oracle.lstm_sequence(Wc, Wa, None, wl.I, wl.H, xs, h0, c0, wl.k_a, wl.T)
+    else:
+        oracle.gru_sequence(Wc, Wa, None, wl.I, wl.H, xs, h0, wl.k_a, wl.T)
+    return wl.steps * b
+
+
+def oracle_sample_plan(wl):
+    """Bounded sample of the workload for the CPU legs: (rows_limit, batch_limit, description)."""
+    if wl.cell == "proj":
+        return 2048, 32, "first 2048 of %d weight rows x first 32 of %d activation vectors (scaled by work)" % (wl.m, wl.batch)
+    if wl.batch > 2:
+        return None, 2, "all %d timesteps for the first 2 of %d sequences" % (wl.steps, wl.batch)
+    return None, None, "the full workload (%d timesteps, batch %d)" % (wl.steps, wl.batch)
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    rows_limit, batch_limit, desc = oracle_sample_plan(wl)
+    Wc, Wa = oracle_setup(wl, rows_limit)
+    ins = synth.inputs(wl)
+    for _ in range(args.warmup):
+        oracle_step(wl, Wc, Wa, ins, batch_limit)
+    units = 0.0
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        units += oracle_step(wl, Wc, Wa, ins, batch_limit)
+    dt = time.perf_counter() - t0
+    value = units / dt if wl.cell != "proj" else units / dt
+    unit = "timesteps/s" if wl.cell != "proj" else "passes/s"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": unit, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(wl, "n/a (CPU)"),
+        "cpu_baseline": {"value": value, "unit": unit, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def workload_config(wl, l2_note):
+    return {
+        "workload": wl.name, "cell": wl.cell, "input": wl.I, "hidden": wl.H, "rows": wl.m, "cols": wl.n,
+        "k_w": wl.k_w, "k_a": wl.k_a, "T": wl.T, "batch": wl.batch, "timesteps": wl.steps,
+        "weights": "N(0,%g^2)" % wl.w_std, "inputs": wl.x_dist, "seed": wl.seed, "l2": l2_note,
+        "parallelism": "independent sequences per GPU (replicas)",
+    }
+
+
+# ---- clocks ----------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid, self.proc, self.lines = uuid, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---- our arm ---------------------------------------------------------------------------------------------
+
+def run_ours(args, wl):
+    import torch
+    from paper_1802_00150_b200 import amq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    stream = torch.cuda.current_stream()
+
+    # inputs: every rank draws its own sequences (seed offset by rank); weights are the same model
+    wl_rank = synth.scaled(wl, seed=wl.seed + 1000 * rank) if rank else wl
+    ins = synth.inputs(wl_rank)
+    W = torch.from_numpy(synth.weights(wl)).to(dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)        # 256 MiB > L2 (126 MB)
+
+    if wl.cell == "proj":
+        acts = torch.from_numpy(ins["acts"]).to(dev)
+        Wcodes = torch.empty((wl.m, wl.k_w, amq.words_per_row(wl.n)), dtype=torch.int32, device=dev)
+        Walpha = torch.empty((wl.m, wl.k_w), dtype=torch.float32, device=dev)
+        y = torch.empty((wl.batch, wl.m), dtype=torch.float32, device=dev)
+
+        def step():
+            amq.quantize(W, wl.k_w, wl.T, codes=Wcodes, coeffs=Walpha)
+            xc, xb = amq.quantize(acts, wl.k_a, wl.T)
+            amq.binary_gemm(Wcodes, Walpha, xc, xb, wl.n, y=y)
+
+        h2d = acts.numel() * 4
+        d2h = 4 * wl.batch
+        acts_host = torch.from_numpy(ins["acts"]).pin_memory()
+        y_host = torch.empty((wl.batch,), dtype=torch.float32).pin_memory()
+
+        def step_e2e():
+            acts.copy_(acts_host, non_blocking=True)
+            step()
+            y_host.copy_(y[:, 0], non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+    else:
+        Wcodes, Walpha = amq.quantize(W, wl.k_w, wl.T)
+        del W
+        x_seq = torch.from_numpy(ins["x_seq"]).to(dev)
+        h0, c0 = torch.from_numpy(ins["h0"]).to(dev), torch.from_numpy(ins["c0"]).to(dev)
+        ws = amq.new_workspace(wl.I, wl.H, wl.batch, wl.k_a)
+        staging = amq.new_host_staging(wl.I, wl.H, wl.batch, wl.steps)
+        h_last, c_last = torch.empty_like(h0), torch.empty_like(c0)
+        xs_host = torch.from_numpy(ins["x_seq"]).pin_memory()
+        h0_host, c0_host = torch.from_numpy(ins["h0"]).pin_memory(), torch.from_numpy(ins["c0"]).pin_memory()
+        hl_host, cl_host = torch.empty_like(h0_host).pin_memory(), torch.empty_like(c0_host).pin_memory()
+        if wl.cell == "lstm":
+            def step():
+                amq.lstm_sequence(Wcodes, Walpha, None, wl.I, wl.H, x_seq, h0, c0, wl.k_a, wl.T, ws,
+                                  h_last=h_last, c_last=c_last)
+
+            def step_e2e():
+                amq.lstm_sequence_host(Wcodes, Walpha, None, wl.I, wl.H, xs_host, h0_host, c0_host, wl.k_a, wl.T,
+                                       ws, staging, hl_host, cl_host)
+            h2d = (xs_host.numel() + 2 * h0_host.numel()) * 4
+            d2h = 2 * h0_host.numel() * 4
+        else:
+            def step():
+                amq.gru_sequence(Wcodes, Walpha, None, wl.I, wl.H, x_seq, h0, wl.k_a, wl.T, ws, h_last=h_last)
+
+            def step_e2e():
+                amq.gru_sequence_host(Wcodes, Walpha, None, wl.I, wl.H, xs_host, h0_host, wl.k_a, wl.T,
+                                      ws, staging, hl_host)
+            h2d = (xs_host.numel() + h0_host.numel()) * 4
+            d2h = h0_host.numel() * 4
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, iters, warmup):
+        """Per-iteration CUDA events on the launching stream; L2 flushed (untimed) before each iteration."""
+        for _ in range(warmup):
+            fn()
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(iters)]
+        stops = [torch.cuda.Event(enable_timing=True) for _ in range(iters)]
+        barrier()
+        launches0 = amq.kernel_launches()
+        for i in range(iters):
+            flush.fill_(i & 0xFF)
+            starts[i].record(stream)
+            fn()
+            stops[i].record(stream)
+        barrier()
+        launches = amq.kernel_launches() - launches0
+        ms = [s.elapsed_time(e) for s, e in zip(starts, stops)]
+        return ms, launches
+
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    if rank == 0:
+        sampler.start()
+    ms, launches = timed(step, args.steps, max(args.warmup, 3))
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = float(sum(ms))
+    ms_e2e, _ = timed(step_e2e, max(3, min(args.steps, 20)), 3)
+    e2e_total_ms = float(sum(ms_e2e))
+    e2e_iters = len(ms_e2e)
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_total_ms = float(t[0]), float(t[1])
+        lt = torch.tensor([launches], device=dev, dtype=torch.int64)
+        dist.all_reduce(lt, op=dist.ReduceOp.SUM)
+        launches = int(lt[0])
+    assert amq.workspace_status(ws) == 0 if wl.cell != "proj" else True
+
+    units = units_per_step(wl)
+    unit = "timesteps/s" if wl.cell != "proj" else "passes/s"
+    value = world * units * args.steps / (total_ms * 1e-3)
+    e2e_value = world * units * e2e_iters / (e2e_total_ms * 1e-3)
+    peak, peak_kind = measured_peaks()
+
+    line = None
+    if rank == 0:
+        step_ms = total_ms / args.steps
+        if wl.cell == "proj":
+            alg_bytes = wl.m * wl.n * 4 + wl.k_w * wl.m * ((wl.n + 31) // 32) * 4 * 2 + wl.batch * wl.m * 4
+            kernel_name = "bulk quantize + binary GEMM (whole step)"
+        else:
+            alg_bytes = algorithmic_bytes_per_timestep(wl) * wl.steps
+            kernel_name = "sequence step chain (quantize + binary product with gate epilogue)"
+        achieved = alg_bytes / (step_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u32 popcount + f32", "data": "synthetic",
+            "config": workload_config(wl, "flushed before every step by an untimed 256 MiB write; inside a step "
+                                          "the packed weights are re-read from L2 by design"),
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": "of " + peak_kind,
+                         "frac_of_nominal_8000": achieved / 8000.0,
+                         "algorithmic_bytes_per_launch": int(alg_bytes),
+                         "traffic": NCU_TRAFFIC_BYTES.get(wl.name)},
+            "us_per_timestep": 1e3 * step_ms / max(wl.steps, 1) if wl.cell != "proj" else None,
+        }
+        if not args.no_extras and world == 1:
+            line["gemv_cold"] = cold_gemv(amq, torch, dev, flush, peak, peak_kind)
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(wl, unit)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line))
+
+
+def cold_gemv(amq, torch, dev, flush, peak, peak_kind):
+    """Batch-1 binary GEMV on packed planes far larger than L2 (HBM-bound): achieved GB/s of packed weights."""
+    m, n, k_w, k_a = 131072, 8192, 2, 2
+    wpr = amq.words_per_row(n)
+    g = torch.Generator(device=dev)
+    g.manual_seed(0)
+    Wcodes = torch.randint(-2 ** 31, 2 ** 31 - 1, (m, k_w, wpr), dtype=torch.int32, device=dev, generator=g)
+    Walpha = torch.rand((m, k_w), device=dev, generator=g) * 0.02
+    x = torch.from_numpy(synth.uniform((1, n), -1, 1, 0, 9)).to(dev)
+    xc, xb = amq.quantize(x, k_a, 2)
+    y = torch.empty((1, m), device=dev)
+    for _ in range(3):
+        amq.binary_gemm(Wcodes, Walpha, xc, xb, n, y=y)
+    times = []
+    for i in range(10):
+        flush.fill_(i)
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        amq.binary_gemm(Wcodes, Walpha, xc, xb, n, y=y)
+        e.record()
+        torch.cuda.synchronize()
+        times.append(s.elapsed_time(e))
+    ms = float(np.median(times))
+    alg = Wcodes.numel() * 4 + Walpha.numel() * 4 + m * 4 + xc.numel() * 4
+    gbs = alg / (ms * 1e-3) / 1e9
+    return {"workload": "batch-1 binary GEMV %dx%d, k_w=%d, k_a=%d, packed planes %d MiB (random bits), cold" % (
+                m, n, k_w, k_a, Wcodes.numel() * 4 >> 20),
+            "ms": ms, "achieved": gbs, "unit": "GB/s", "peak": peak, "frac": gbs / peak, "peak_kind": "of " + peak_kind,
+            "frac_of_nominal_8000": gbs / 8000.0, "algorithmic_bytes": int(alg)}
+
+
+def cpu_baseline(wl, unit):
+    """The oracle, as it stands, on one host core, on a bounded sample of the same workload (~10-30 s)."""
+    rows_limit, batch_limit, desc = oracle_sample_plan(wl)
+    Wc, Wa = oracle_setup(wl, rows_limit)
+    ins = synth.inputs(wl)
+    units, t0 = 0.0, time.perf_counter()
+    reps = 0
+    while True:
+        units += oracle_step(wl, Wc, Wa, ins, batch_limit)
+        reps += 1
+        if time.perf_counter() - t0 > 10.0 or reps >= 200:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": units / dt, "unit": unit, "cores": 1, "kind": "oracle",
+            "sample": "%d x %s; fp64, single thread; weight quantization not timed" % (reps, desc)}
+
+
+def main():
+    args = parse_args()
+    wl = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

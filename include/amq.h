@@ -1,0 +1,205 @@
+/*
+ * amq.h -- C ABI of the B200 (sm_100a) library for alternating multi-bit quantization:
+ * row-wise quantizer, bit-plane packing, binary (XNOR / bit-count) matrix product, and quantized
+ * LSTM / GRU steps with the gate arithmetic fused behind the product.
+ *
+ * Paper: "Alternating Multi-bit Quantization for Recurrent Neural Networks".  Each entry point cites
+ * the passage that defines what it computes.
+ *
+ * General rules
+ *   - Unless an argument is documented as HOST, every pointer is a DEVICE pointer owned by the caller
+ *     and valid on the device that is current when the call is made.  The library keeps no pointer
+ *     after the work it enqueued has finished.  It allocates no device memory: calls that need scratch
+ *     take a caller-provided workspace whose size comes from the matching *_workspace_bytes function.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue work
+ *     and return; they do not synchronise, except the *_host variants, which return after their
+ *     results are in host memory.
+ *   - Return value: AMQ_OK or a negative amq_status.  Invalid arguments are detected on the host before
+ *     anything is launched; nothing traps or aborts.  Faults that can only be seen on the device
+ *     (a bounded wait that ran out) are written to a status word at the start of the workspace and are
+ *     read with amq_workspace_status.
+ *   - Layouts are row-major.  1 <= k <= 4 for every bit count; n >= 1.
+ *
+ * Packed codes ("k planes of 32-bit words"):
+ *   a length-n vector quantized to k bits is stored as k bit-planes, plane i (i = 0..k-1, the paper's
+ *   b_{i+1}) in wpr = amq_words_per_row(n) = 4 * ceil(n / 128) consecutive uint32 words; bit j of word q
+ *   holds element 32q + j; bit 1 means +1, bit 0 means -1; bits at positions >= n are 0.
+ *   A matrix of `rows` vectors is codes[row][plane][wpr] with coefficients coeffs[row][k] (fp32).
+ *   Code buffers must be 16-byte aligned (they are read with 128-bit loads).
+ */
+#ifndef AMQ_H
+#define AMQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define AMQ_API __attribute__((visibility("default")))
+#else
+#define AMQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int amq_status;
+enum {
+    AMQ_OK = 0,
+    AMQ_ERR_INVALID_ARG = -1,   /* NULL where data is required, non-positive size, ld too small, aliasing */
+    AMQ_ERR_UNSUPPORTED = -2,   /* k outside 1..4, T < 0, n beyond AMQ_MAX_N, batch beyond a kernel's limit */
+    AMQ_ERR_ALIGNMENT = -3,     /* a code or workspace pointer is not 16-byte aligned */
+    AMQ_ERR_WORKSPACE = -4,     /* workspace NULL or smaller than *_workspace_bytes */
+    AMQ_ERR_CUDA = -5,          /* a CUDA runtime call failed; see amq_last_cuda_error */
+    AMQ_ERR_TIMEOUT = -6        /* a bounded device-side wait ran out (reported by amq_workspace_status) */
+};
+
+#define AMQ_MAX_K 4
+#define AMQ_MAX_N 8192          /* longest vector the row quantizer accepts */
+
+/* Text for a status code (static storage, never NULL). */
+AMQ_API const char* amq_status_string(amq_status s);
+/* cudaError_t (as int) of the most recent failing CUDA call made by this library on this thread; 0 if none. */
+AMQ_API int amq_last_cuda_error(void);
+
+/* Number of kernels this library has enqueued so far in this process (all threads, all streams). */
+AMQ_API unsigned long long amq_kernel_launches(void);
+
+/* 4 * ceil(n / 128): 32-bit words per packed plane. */
+AMQ_API int amq_words_per_row(int n);
+/* rows * k * amq_words_per_row(n) * 4: bytes of a packed code buffer. */
+AMQ_API size_t amq_codes_bytes(int rows, int n, int k);
+
+/*
+ * Row-wise alternating multi-bit quantization (Algorithm 2, with the greedy initialisation of Eq. 3-4,
+ * the least-squares refit of Eq. 5 and the binary-search-tree code assignment of Algorithm 1).
+ * Each of the `rows` rows of x is quantized on its own ("row by row", Sec. 4); the same call quantizes
+ * weights offline and activations on-line.
+ *   x       [rows][ldx] fp32, ldx >= n (elements).
+ *   k, T    bits and alternating cycles (T >= 0; T = 0 returns the greedy solution).
+ *   codes   [rows][k][wpr] uint32 out;  coeffs [rows][k] fp32 out.
+ * Readings where the paper is silent: sign(0) = +1; the level table is sorted by (value, code index)
+ * with plane 0 the most significant code bit; a refit whose k x k system has a pivot below 1e-9 * n
+ * (Gaussian elimination with partial pivoting, in double) is skipped and keeps the previous coefficients.
+ * Sums over a row are accumulated in fp32 per thread and in fp64 across threads; the solve is fp64;
+ * levels, thresholds and comparisons are fp32.
+ */
+AMQ_API amq_status amq_quantize(const float* x, int rows, int n, int ldx, int k, int T,
+                        uint32_t* codes, float* coeffs, void* stream);
+
+/*
+ * Pack sign planes given as floats into the bit layout above (storage for the XNOR / bit-count
+ * product, Appendix A).  planes [rows][k][n] fp32, value >= 0 -> bit 1.  codes [rows][k][wpr] out.
+ */
+AMQ_API amq_status amq_pack(const float* planes, int rows, int n, int k, uint32_t* codes, void* stream);
+
+/* Reconstruction of Eq. 2: xhat[row][t] = sum_i coeffs[row][i] * (+1 or -1).  xhat [rows][n] fp32 out. */
+AMQ_API amq_status amq_unpack(const uint32_t* codes, const float* coeffs, int rows, int n, int k,
+                      float* xhat, void* stream);
+
+/*
+ * Integer partials of the quantized product (Sec. 4, Fig. 3; XNOR then bit count, Appendix A):
+ *   D[b][r][i][j] = B_i[r,:] . x_j[b] = n - 2 * popcount(Wcodes[r][i] xor xcodes[b][j]),   int32.
+ * Wcodes [m][k_w][wpr], xcodes [batch][k_a][wpr], D [batch][m][k_w][k_a] out.  Exact.
+ */
+AMQ_API amq_status amq_binary_dots(const uint32_t* Wcodes, int m, int n, int k_w,
+                           const uint32_t* xcodes, int batch, int k_a, int32_t* D, void* stream);
+
+/*
+ * Quantized matrix product (Sec. 4: binary product first, then the row-wise coefficients; the stacked
+ * form of Fig. 3, right, for batch > 1):
+ *   y[b][r] = sum_i sum_j Walpha[r][i] * xbeta[b][j] * D[b][r][i][j] + bias[r].
+ * Walpha [m][k_w], xbeta [batch][k_a], bias [m] or NULL, y [batch][ldy] fp32 out, ldy >= m.
+ * The integer partials are exact; the combination is fp32.
+ */
+AMQ_API amq_status amq_binary_gemm(const uint32_t* Wcodes, const float* Walpha, int m, int n, int k_w,
+                           const uint32_t* xcodes, const float* xbeta, int batch, int k_a,
+                           const float* bias, float* y, int ldy, void* stream);
+
+/* Scratch for the cell calls below (steps and sequences), in bytes; 0 on invalid arguments. */
+AMQ_API size_t amq_cell_workspace_bytes(int I, int H, int batch, int k_a);
+/* Additional device staging needed by the *_host variants (x_seq, states and results), in bytes. */
+AMQ_API size_t amq_cell_host_staging_bytes(int I, int H, int batch, int steps);
+
+/*
+ * One quantized LSTM step (Eq. 6) for `batch` independent sequences.
+ *   W: the stacked gate matrix, 4H rows in the order i, f, o, g (the order Eq. 6 prints), I + H columns
+ *      (input part first), quantized offline row by row: Wcodes [4H][k_w][wpr(I+H)], Walpha [4H][k_w].
+ *   z = [x ; h_in] is quantized on-line as one vector with k_a bits and T cycles, then
+ *   p = W_hat z_hat + bias;  i, f, o = logistic(p);  g = tanh(p);  c_out = f*c_in + i*g;  h_out = o*tanh(c_out).
+ *   bias [4H] (b_i + b_h of Eq. 6 summed) or NULL.  x [batch][I]; h_in, c_in, h_out, c_out [batch][H] fp32.
+ *   h_out must not alias h_in; c_out may alias c_in.
+ */
+AMQ_API amq_status amq_lstm_step(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                         int I, int H, int k_w,
+                         const float* x, const float* h_in, const float* c_in, int batch, int k_a, int T,
+                         float* h_out, float* c_out,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * One quantized GRU step.  The paper names the GRU (Sec. 1, Sec. 5) without printing its equations;
+ * this library computes the "linear before reset" form:
+ *   W: 3H rows in the order r, z, n;  p = W_hat z_hat with z_hat the quantized [x ; h_in];
+ *   for the n rows the product is kept in two column segments, p_nx over [0, I) and p_nh over [I, I+H);
+ *   r = logistic(p_r + b_r);  z = logistic(p_z + b_z);  cand = tanh(p_nx + b_nx + r * (p_nh + b_nh));
+ *   h_out = (1 - z) * cand + z * h_in.
+ *   bias [4H] = [b_r ; b_z ; b_nx ; b_nh] or NULL.  h_out must not alias h_in.
+ */
+AMQ_API amq_status amq_gru_step(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                        int I, int H, int k_w,
+                        const float* x, const float* h_in, int batch, int k_a, int T,
+                        float* h_out,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * `steps` consecutive steps without returning to the host ("RNNs can only be executed sequentially",
+ * Sec. 1: step t+1 consumes h_t).  x_seq [steps][batch][I]; h0, c0 [batch][H];
+ * h_seq [steps][batch][H] out or NULL; h_last, c_last [batch][H] out.  Outputs must not alias inputs.
+ */
+AMQ_API amq_status amq_lstm_sequence(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                             int I, int H, int k_w,
+                             const float* x_seq, int steps, const float* h0, const float* c0,
+                             int batch, int k_a, int T,
+                             float* h_seq, float* h_last, float* c_last,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+AMQ_API amq_status amq_gru_sequence(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                            int I, int H, int k_w,
+                            const float* x_seq, int steps, const float* h0,
+                            int batch, int k_a, int T,
+                            float* h_seq, float* h_last,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The sequence calls with HOST activations and results: x_seq, h0, c0 are read from host memory
+ * (pinned memory makes the copies asynchronous) into `staging`, the sequence runs, and h_last / c_last
+ * (and h_seq when not NULL) are copied back to host memory; the call returns after the stream has
+ * drained.  Weights, bias, workspace and staging (amq_cell_host_staging_bytes) stay DEVICE pointers.
+ */
+AMQ_API amq_status amq_lstm_sequence_host(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                                  int I, int H, int k_w,
+                                  const float* x_seq_host, int steps, const float* h0_host, const float* c0_host,
+                                  int batch, int k_a, int T,
+                                  float* h_seq_host, float* h_last_host, float* c_last_host,
+                                  void* workspace, size_t workspace_bytes,
+                                  void* staging, size_t staging_bytes, void* stream);
+
+AMQ_API amq_status amq_gru_sequence_host(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                                 int I, int H, int k_w,
+                                 const float* x_seq_host, int steps, const float* h0_host,
+                                 int batch, int k_a, int T,
+                                 float* h_seq_host, float* h_last_host,
+                                 void* workspace, size_t workspace_bytes,
+                                 void* staging, size_t staging_bytes, void* stream);
+
+/*
+ * Synchronises `stream`, then reads the status word at the start of a cell workspace: AMQ_OK, or
+ * AMQ_ERR_TIMEOUT if a bounded device-side wait gave up during a call that used this workspace.
+ * The word is cleared by the next cell call.
+ */
+AMQ_API amq_status amq_workspace_status(const void* workspace, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMQ_H */

@@ -1,0 +1,223 @@
+// Quantized LSTM / GRU steps and sequences (Eq. 6; on-line quantization of the activation, Sec. 4):
+// each step is the row quantizer on z = [x ; h] followed by the binary product with the fused gate
+// epilogue.  No step returns to the host; a sequence is enqueued as one chain on the caller's stream.
+#include "amq_common.cuh"
+
+namespace amq {
+
+namespace {
+
+struct CellCall {
+    const uint32_t* Wcodes; const float* Walpha; const float* bias;
+    int I, H, k_w, batch, k_a, T;
+    bool gru;
+};
+
+amq_status validate(const CellCall& c, const void* workspace, size_t workspace_bytes)
+{
+    if (!c.Wcodes || !c.Walpha || c.I < 0 || c.H < 1 || c.batch < 0) return AMQ_ERR_INVALID_ARG;
+    if (!valid_k(c.k_w) || !valid_k(c.k_a) || c.T < 0 || c.I + c.H > AMQ_MAX_N) return AMQ_ERR_UNSUPPORTED;
+    if (!aligned16(c.Wcodes)) return AMQ_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < amq_cell_workspace_bytes(c.I, c.H, c.batch, c.k_a)) return AMQ_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return AMQ_ERR_ALIGNMENT;
+    return AMQ_OK;
+}
+
+// quantize z = [x ; h_in] into the workspace, then product + gates
+amq_status enqueue_step(const CellCall& c, const CellWorkspace& ws, const float* x, const float* h_in,
+                        const float* c_in, float* h_out, float* c_out, cudaStream_t st)
+{
+    amq_status s = launch_quantize(x, c.I, c.I, h_in, c.H, c.H, c.batch, c.k_a, c.T, ws.zcodes, ws.zbeta, st);
+    if (s != AMQ_OK) return s;
+    GemmArgs a{};
+    a.Wcodes = c.Wcodes; a.Walpha = c.Walpha; a.m = (c.gru ? 3 : 4) * c.H; a.n = c.I + c.H; a.k_w = c.k_w;
+    a.xcodes = ws.zcodes; a.xbeta = ws.zbeta; a.batch = c.batch; a.k_a = c.k_a;
+    a.bias = c.bias; a.epilogue = c.gru ? EPI_GRU : EPI_LSTM;
+    a.I = c.I; a.H = c.H; a.h_in = h_in; a.c_in = c_in; a.h_out = h_out; a.c_out = c_out;
+    return launch_binary_gemm(a, st);
+}
+
+amq_status enqueue_sequence(const CellCall& c, const CellWorkspace& ws, const float* x_seq, int steps,
+                            const float* h0, const float* c0, float* h_seq, float* h_last, float* c_last,
+                            cudaStream_t st)
+{
+    const size_t state_bytes = (size_t)c.batch * c.H * sizeof(float);
+    AMQ_CUDA_TRY(cudaMemsetAsync(ws.status, 0, 256, st));
+    if (!c.gru) AMQ_CUDA_TRY(cudaMemcpyAsync(ws.c, c0, state_bytes, cudaMemcpyDeviceToDevice, st));
+    const float* h_prev = h0;
+    for (int s = 0; s < steps; ++s) {
+        float* h_next = h_seq ? h_seq + (size_t)s * c.batch * c.H : ws.h[s & 1];
+        const float* x = x_seq + (size_t)s * c.batch * c.I;
+        amq_status r = enqueue_step(c, ws, x, h_prev, ws.c, h_next, ws.c, st);
+        if (r != AMQ_OK) return r;
+        h_prev = h_next;
+    }
+    AMQ_CUDA_TRY(cudaMemcpyAsync(h_last, h_prev, state_bytes, cudaMemcpyDeviceToDevice, st));
+    if (!c.gru) AMQ_CUDA_TRY(cudaMemcpyAsync(c_last, ws.c, state_bytes, cudaMemcpyDeviceToDevice, st));
+    return AMQ_OK;
+}
+
+amq_status sequence_entry(const CellCall& c, const float* x_seq, int steps, const float* h0, const float* c0,
+                          float* h_seq, float* h_last, float* c_last,
+                          void* workspace, size_t workspace_bytes, cudaStream_t st)
+{
+    amq_status s = validate(c, workspace, workspace_bytes);
+    if (s != AMQ_OK) return s;
+    if (steps < 0 || !h0 || !h_last || (!c.gru && (!c0 || !c_last)) || (steps > 0 && c.I > 0 && !x_seq))
+        return AMQ_ERR_INVALID_ARG;
+    if (h_last == h0 || (!c.gru && c_last == c0)) return AMQ_ERR_INVALID_ARG;
+    if (c.batch == 0) return AMQ_OK;
+    CellWorkspace ws = carve_cell_workspace(workspace, c.I, c.H, c.batch, c.k_a);
+    return enqueue_sequence(c, ws, x_seq, steps, h0, c0, h_seq, h_last, c_last, st);
+}
+
+struct HostStaging {
+    float* x_seq; float* h0; float* c0; float* h_seq; float* h_last; float* c_last;
+    size_t bytes;
+};
+
+HostStaging carve_staging(void* base, int I, int H, int batch, int steps)
+{
+    HostStaging s;
+    char* p = static_cast<char*>(base);
+    size_t off = 0;
+    const size_t state = round_up((size_t)batch * H * 4, 256);
+    s.x_seq = reinterpret_cast<float*>(p + off);  off += round_up((size_t)steps * batch * I * 4, 256);
+    s.h0 = reinterpret_cast<float*>(p + off);     off += state;
+    s.c0 = reinterpret_cast<float*>(p + off);     off += state;
+    s.h_seq = reinterpret_cast<float*>(p + off);  off += round_up((size_t)steps * batch * H * 4, 256);
+    s.h_last = reinterpret_cast<float*>(p + off); off += state;
+    s.c_last = reinterpret_cast<float*>(p + off); off += state;
+    s.bytes = off;
+    return s;
+}
+
+amq_status sequence_host_entry(const CellCall& c, const float* x_seq_host, int steps, const float* h0_host,
+                               const float* c0_host, float* h_seq_host, float* h_last_host, float* c_last_host,
+                               void* workspace, size_t workspace_bytes, void* staging, size_t staging_bytes,
+                               cudaStream_t st)
+{
+    amq_status s = validate(c, workspace, workspace_bytes);
+    if (s != AMQ_OK) return s;
+    if (steps < 0 || !h0_host || !h_last_host || (!c.gru && (!c0_host || !c_last_host)) ||
+        (steps > 0 && c.I > 0 && !x_seq_host))
+        return AMQ_ERR_INVALID_ARG;
+    if (!staging || staging_bytes < amq_cell_host_staging_bytes(c.I, c.H, c.batch, steps)) return AMQ_ERR_WORKSPACE;
+    if (!aligned16(staging)) return AMQ_ERR_ALIGNMENT;
+    if (c.batch == 0) return AMQ_OK;
+    CellWorkspace ws = carve_cell_workspace(workspace, c.I, c.H, c.batch, c.k_a);
+    HostStaging hs = carve_staging(staging, c.I, c.H, c.batch, steps);
+    const size_t state_bytes = (size_t)c.batch * c.H * sizeof(float);
+    const size_t x_bytes = (size_t)steps * c.batch * c.I * sizeof(float);
+    if (x_bytes) AMQ_CUDA_TRY(cudaMemcpyAsync(hs.x_seq, x_seq_host, x_bytes, cudaMemcpyHostToDevice, st));
+    AMQ_CUDA_TRY(cudaMemcpyAsync(hs.h0, h0_host, state_bytes, cudaMemcpyHostToDevice, st));
+    if (!c.gru) AMQ_CUDA_TRY(cudaMemcpyAsync(hs.c0, c0_host, state_bytes, cudaMemcpyHostToDevice, st));
+    s = enqueue_sequence(c, ws, hs.x_seq, steps, hs.h0, hs.c0, h_seq_host ? hs.h_seq : nullptr, hs.h_last,
+                         hs.c_last, st);
+    if (s != AMQ_OK) return s;
+    if (h_seq_host && steps > 0)
+        AMQ_CUDA_TRY(cudaMemcpyAsync(h_seq_host, hs.h_seq, (size_t)steps * state_bytes, cudaMemcpyDeviceToHost, st));
+    AMQ_CUDA_TRY(cudaMemcpyAsync(h_last_host, hs.h_last, state_bytes, cudaMemcpyDeviceToHost, st));
+    if (!c.gru) AMQ_CUDA_TRY(cudaMemcpyAsync(c_last_host, hs.c_last, state_bytes, cudaMemcpyDeviceToHost, st));
+    AMQ_CUDA_TRY(cudaStreamSynchronize(st));
+    return AMQ_OK;
+}
+
+}  // namespace
+}  // namespace amq
+
+extern "C" {
+
+size_t amq_cell_workspace_bytes(int I, int H, int batch, int k_a)
+{
+    if (I < 0 || H < 1 || batch < 0 || !amq::valid_k(k_a)) return 0;
+    return amq::carve_cell_workspace(nullptr, I, H, batch, k_a).bytes;
+}
+
+size_t amq_cell_host_staging_bytes(int I, int H, int batch, int steps)
+{
+    if (I < 0 || H < 1 || batch < 0 || steps < 0) return 0;
+    return amq::carve_staging(nullptr, I, H, batch, steps).bytes;
+}
+
+amq_status amq_lstm_step(const uint32_t* Wcodes, const float* Walpha, const float* bias, int I, int H, int k_w,
+                         const float* x, const float* h_in, const float* c_in, int batch, int k_a, int T,
+                         float* h_out, float* c_out, void* workspace, size_t workspace_bytes, void* stream)
+{
+    amq::CellCall c{Wcodes, Walpha, bias, I, H, k_w, batch, k_a, T, false};
+    amq_status s = amq::validate(c, workspace, workspace_bytes);
+    if (s != AMQ_OK) return s;
+    if (!h_in || !c_in || !h_out || !c_out || (I > 0 && !x) || h_out == h_in) return AMQ_ERR_INVALID_ARG;
+    if (batch == 0) return AMQ_OK;
+    amq::CellWorkspace ws = amq::carve_cell_workspace(workspace, I, H, batch, k_a);
+    AMQ_CUDA_TRY(cudaMemsetAsync(ws.status, 0, 256, (cudaStream_t)stream));
+    return amq::enqueue_step(c, ws, x, h_in, c_in, h_out, c_out, (cudaStream_t)stream);
+}
+
+amq_status amq_gru_step(const uint32_t* Wcodes, const float* Walpha, const float* bias, int I, int H, int k_w,
+                        const float* x, const float* h_in, int batch, int k_a, int T,
+                        float* h_out, void* workspace, size_t workspace_bytes, void* stream)
+{
+    amq::CellCall c{Wcodes, Walpha, bias, I, H, k_w, batch, k_a, T, true};
+    amq_status s = amq::validate(c, workspace, workspace_bytes);
+    if (s != AMQ_OK) return s;
+    if (!h_in || !h_out || (I > 0 && !x) || h_out == h_in) return AMQ_ERR_INVALID_ARG;
+    if (batch == 0) return AMQ_OK;
+    amq::CellWorkspace ws = amq::carve_cell_workspace(workspace, I, H, batch, k_a);
+    AMQ_CUDA_TRY(cudaMemsetAsync(ws.status, 0, 256, (cudaStream_t)stream));
+    return amq::enqueue_step(c, ws, x, h_in, nullptr, h_out, nullptr, (cudaStream_t)stream);
+}
+
+amq_status amq_lstm_sequence(const uint32_t* Wcodes, const float* Walpha, const float* bias, int I, int H, int k_w,
+                             const float* x_seq, int steps, const float* h0, const float* c0,
+                             int batch, int k_a, int T, float* h_seq, float* h_last, float* c_last,
+                             void* workspace, size_t workspace_bytes, void* stream)
+{
+    amq::CellCall c{Wcodes, Walpha, bias, I, H, k_w, batch, k_a, T, false};
+    return amq::sequence_entry(c, x_seq, steps, h0, c0, h_seq, h_last, c_last, workspace, workspace_bytes,
+                               (cudaStream_t)stream);
+}
+
+amq_status amq_gru_sequence(const uint32_t* Wcodes, const float* Walpha, const float* bias, int I, int H, int k_w,
+                            const float* x_seq, int steps, const float* h0, int batch, int k_a, int T,
+                            float* h_seq, float* h_last, void* workspace, size_t workspace_bytes, void* stream)
+{
+    amq::CellCall c{Wcodes, Walpha, bias, I, H, k_w, batch, k_a, T, true};
+    return amq::sequence_entry(c, x_seq, steps, h0, nullptr, h_seq, h_last, nullptr, workspace, workspace_bytes,
+                               (cudaStream_t)stream);
+}
+
+amq_status amq_lstm_sequence_host(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                                  int I, int H, int k_w, const float* x_seq_host, int steps,
+                                  const float* h0_host, const float* c0_host, int batch, int k_a, int T,
+                                  float* h_seq_host, float* h_last_host, float* c_last_host,
+                                  void* workspace, size_t workspace_bytes, void* staging, size_t staging_bytes,
+                                  void* stream)
+{
+    amq::CellCall c{Wcodes, Walpha, bias, I, H, k_w, batch, k_a, T, false};
+    return amq::sequence_host_entry(c, x_seq_host, steps, h0_host, c0_host, h_seq_host, h_last_host, c_last_host,
+                                    workspace, workspace_bytes, staging, staging_bytes, (cudaStream_t)stream);
+}
+
+amq_status amq_gru_sequence_host(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                                 int I, int H, int k_w, const float* x_seq_host, int steps,
+                                 const float* h0_host, int batch, int k_a, int T,
+                                 float* h_seq_host, float* h_last_host,
+                                 void* workspace, size_t workspace_bytes, void* staging, size_t staging_bytes,
+                                 void* stream)
+{
+    amq::CellCall c{Wcodes, Walpha, bias, I, H, k_w, batch, k_a, T, true};
+    return amq::sequence_host_entry(c, x_seq_host, steps, h0_host, nullptr, h_seq_host, h_last_host, nullptr,
+                                    workspace, workspace_bytes, staging, staging_bytes, (cudaStream_t)stream);
+}
+
+amq_status amq_workspace_status(const void* workspace, void* stream)
+{
+    if (!workspace) return AMQ_ERR_INVALID_ARG;
+    AMQ_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    uint32_t word = 0;
+    AMQ_CUDA_TRY(cudaMemcpy(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost));
+    return word == 0 ? AMQ_OK : AMQ_ERR_TIMEOUT;
+}
+
+}  // extern "C"

@@ -1,0 +1,89 @@
+// Shared host/device helpers of the CUDA library (status handling, sizes, small device utilities).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "amq.h"
+
+namespace amq {
+
+// Last failing CUDA call of this thread (read through amq_last_cuda_error).
+extern thread_local int g_last_cuda_error;
+
+inline amq_status cuda_fail(cudaError_t e)
+{
+    g_last_cuda_error = (int)e;
+    return AMQ_ERR_CUDA;
+}
+
+#define AMQ_CUDA_TRY(expr)                                    \
+    do {                                                      \
+        cudaError_t amq_e_ = (expr);                          \
+        if (amq_e_ != cudaSuccess) return ::amq::cuda_fail(amq_e_); \
+    } while (0)
+
+// Kernels enqueued by this library (read through amq_kernel_launches).
+extern unsigned long long g_kernel_launches;
+
+#define AMQ_LAUNCH_CHECK()                               \
+    do {                                                 \
+        __atomic_fetch_add(&::amq::g_kernel_launches, 1ull, __ATOMIC_RELAXED); \
+        AMQ_CUDA_TRY(cudaGetLastError());                \
+    } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool valid_k(int k) { return k >= 1 && k <= AMQ_MAX_K; }
+inline int words_per_row(int n) { return 4 * ((n + 127) / 128); }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Layout of a cell workspace: [status block][z codes][z coefficients][h ping][h pong][c].
+struct CellWorkspace {
+    uint32_t* status;   // 64 words: [0] status, [1..] barrier counters
+    uint32_t* zcodes;   // [batch][k_a][wpr]
+    float* zbeta;       // [batch][k_a]
+    float* h[2];        // [batch][H] each
+    float* c;           // [batch][H]
+    size_t bytes;
+};
+
+inline CellWorkspace carve_cell_workspace(void* base, int I, int H, int batch, int k_a)
+{
+    CellWorkspace w;
+    char* p = static_cast<char*>(base);
+    size_t off = 0;
+    w.status = reinterpret_cast<uint32_t*>(p + off);            off += 256;
+    w.zcodes = reinterpret_cast<uint32_t*>(p + off);            off += round_up((size_t)batch * k_a * words_per_row(I + H) * 4, 256);
+    w.zbeta = reinterpret_cast<float*>(p + off);                off += round_up((size_t)batch * k_a * 4, 256);
+    w.h[0] = reinterpret_cast<float*>(p + off);                 off += round_up((size_t)batch * H * 4, 256);
+    w.h[1] = reinterpret_cast<float*>(p + off);                 off += round_up((size_t)batch * H * 4, 256);
+    w.c = reinterpret_cast<float*>(p + off);                    off += round_up((size_t)batch * H * 4, 256);
+    w.bytes = off;
+    return w;
+}
+
+// ---- launchers implemented in the .cu files (device pointers, already validated) -----------------------
+
+// Quantize `rows` vectors; element t of row r is src0[r*ld0 + t] for t < n0, else src1[r*ld1 + t - n0].
+amq_status launch_quantize(const float* src0, int ld0, int n0, const float* src1, int ld1, int n1,
+                           int rows, int k, int T, uint32_t* codes, float* coeffs, cudaStream_t st);
+
+enum Epilogue { EPI_DOTS = 0, EPI_Y = 1, EPI_LSTM = 2, EPI_GRU = 3 };
+
+struct GemmArgs {
+    const uint32_t* Wcodes; const float* Walpha; int m, n, k_w;
+    const uint32_t* xcodes; const float* xbeta; int batch, k_a;
+    const float* bias;
+    int epilogue;
+    // EPI_DOTS
+    int32_t* D;
+    // EPI_Y
+    float* y; int ldy;
+    // EPI_LSTM / EPI_GRU
+    int I, H;
+    const float* h_in; const float* c_in; float* h_out; float* c_out;
+};
+
+amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st);
+
+}  // namespace amq

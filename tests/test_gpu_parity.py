@@ -1,0 +1,324 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs.
+Tolerances and the staged protocol are in tests/parity.py."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+from paper_1802_00150_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def amq():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    from paper_1802_00150_b200 import amq as binding
+    return binding
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda()
+
+
+def codes_np(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def codes_dev(c):
+    return torch.from_numpy(np.ascontiguousarray(c).view(np.int32)).cuda()
+
+
+def gpu_quantize_fn(amq):
+    def fn(x, k, T):
+        codes, coeffs = amq.quantize(dev(x), k, T)
+        torch.cuda.synchronize()
+        return codes_np(codes), coeffs.cpu().numpy()
+    return fn
+
+
+# ---- quantizer -------------------------------------------------------------------------------------------
+
+QUANT_CASES = [
+    # rows, n, k, T, distribution   (spans the warp-per-row and CTA-per-row kernels, ragged tails, every k)
+    (64, 600, 2, 2, "uniform"),
+    (37, 1024, 3, 2, "normal"),
+    (16, 2048, 2, 2, "normal"),
+    (9, 4096, 3, 2, "normal"),
+    (3, 8192, 2, 2, "normal"),
+    (5, 8191, 4, 2, "uniform"),
+    (1500, 300, 2, 2, "normal"),
+    (1200, 200, 4, 2, "normal"),
+    (1100, 1000, 3, 3, "heavy"),
+    (1030, 2000, 1, 2, "normal"),
+    (7, 1, 2, 2, "normal"),
+    (7, 31, 3, 2, "normal"),
+    (7, 33, 2, 2, "normal"),
+    (7, 127, 4, 2, "normal"),
+    (7, 129, 2, 1, "normal"),
+    (4, 700, 2, 0, "uniform"),
+    (4, 700, 3, 5, "uniform"),
+]
+
+
+def draw(dist, shape, seed):
+    if dist == "uniform":
+        return synth.uniform(shape, -1, 1, seed, 1)
+    if dist == "normal":
+        return synth.normal(shape, 0.03, seed, 1)
+    u = synth.uniform01(int(np.prod(shape)), seed, 2).reshape(shape)
+    g = synth.normal(shape, 1.0, seed, 3)
+    return np.where(u < 0.9, 0.01 * g, 10.0 + g).astype(np.float32)
+
+
+@pytest.mark.parametrize("rows,n,k,T,dist", QUANT_CASES)
+def test_quantize_matches_oracle(amq, rows, n, k, T, dist):
+    x = draw(dist, (rows, n), 100 + n + k)
+    stats = parity.compare_quantizer(x, k, T, gpu_quantize_fn(amq))
+    print(stats)
+
+
+def test_quantize_degenerate_rows(amq):
+    n = 300
+    x = synth.normal((8, n), 1.0, 5, 1)
+    x[0] = 0.0                     # all-zero vector: coefficients 0, all bits +1, no NaN
+    x[1] = 0.25                    # constant
+    x[2] = np.where(np.arange(n) % 2 == 0, 0.5, -0.5)        # one magnitude: second plane is free
+    x[3, : n // 2] = x[3, n // 2: 2 * (n // 2)]              # duplicated values
+    x[4] = np.round(x[4] * 2) / 2                            # many exact ties
+    x[5] = -0.0
+    for k in (1, 2, 3, 4):
+        codes, coeffs = amq.quantize(dev(x), k, 2)
+        xhat = amq.unpack(codes, coeffs, n).cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(coeffs.cpu().numpy()))
+        c = codes_np(codes)
+        assert parity.pad_bits_zero(c, n)
+        assert np.all(parity.unpack_rows(c, n)[0] == 1) and np.all(coeffs.cpu().numpy()[0] == 0)
+        assert np.all(parity.unpack_rows(c, n)[5] == 1)
+        for r in range(8):
+            o_alpha, o_b = oracle.quantize(x[r].astype(np.float64), k, 2)
+            rec = oracle.reconstruct(o_alpha, o_b)
+            scale = np.abs(o_alpha).sum() + 1e-30
+            # compare reconstructions (several codes are correct when levels coincide)
+            mism = np.abs(rec - xhat[r]) > 2e-4 * scale
+            assert mism.mean() <= 0.01, (k, r, mism.sum())
+
+
+def test_quantize_strided_rows_and_reuse_of_outputs(amq):
+    big = dev(synth.normal((6, 1000), 1.0, 9, 1))
+    view = big[:, 100:700]                      # ldx = 1000, n = 600
+    codes, coeffs = amq.quantize(view, 2, 2)
+    codes2, coeffs2 = amq.quantize(view.contiguous(), 2, 2)
+    assert torch.equal(codes, codes2) and torch.equal(coeffs, coeffs2)
+    # determinism: same input, same bits, also on another stream
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        codes3, coeffs3 = amq.quantize(view, 2, 2)
+    s.synchronize()
+    assert torch.equal(codes, codes3) and torch.equal(coeffs, coeffs3)
+
+
+# ---- pack / unpack ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("rows,n,k", [(3, 1, 1), (5, 33, 2), (4, 600, 3), (2, 2048, 4), (1, 129, 2)])
+def test_pack_unpack(amq, rows, n, k):
+    planes = np.where(synth.uniform01(rows * k * n, 3, n).reshape(rows, k, n) < 0.5, -1.0, 1.0).astype(np.float32)
+    planes[0, 0, 0] = 0.0           # zero counts as +1
+    codes = codes_np(amq.pack(dev(planes)))
+    want = np.stack([oracle.pack_planes(np.where(planes[r] >= 0, 1, -1)) for r in range(rows)])
+    assert np.array_equal(codes, want)
+    coeffs = synth.normal((rows, k), 1.0, 4, n)
+    xhat = amq.unpack(codes_dev(codes), dev(coeffs), n).cpu().numpy()
+    ref = np.stack([oracle.reconstruct(coeffs[r], np.where(planes[r] >= 0, 1, -1)) for r in range(rows)])
+    assert np.allclose(xhat, ref, rtol=1e-6, atol=1e-6)
+
+
+# ---- binary product --------------------------------------------------------------------------------------
+
+GEMM_CASES = [
+    # m, n, k_w, k_a, batch
+    (1200, 600, 2, 2, 1),
+    (130, 2048, 3, 3, 64),
+    (97, 4096, 2, 3, 37),
+    (64, 1024, 3, 2, 33),
+    (50, 129, 4, 4, 5),
+    (33, 31, 1, 1, 3),
+    (257, 300, 1, 4, 17),
+    (40, 8192, 2, 2, 2),
+]
+
+
+@pytest.mark.parametrize("m,n,kw,ka,batch", GEMM_CASES)
+def test_dots_bit_exact_and_product_within_tolerance(amq, m, n, kw, ka, batch):
+    W = synth.normal((m, n), 0.03, 20 + m, 1).astype(np.float64)
+    X = synth.uniform((batch, n), -1, 1, 20 + m, 2).astype(np.float64)
+    bias = synth.normal((m,), 0.1, 20 + m, 3)
+    Wc, Wa = oracle.quantize_rows(W, kw, 2)
+    Xc, Xb = oracle.quantize_rows(X, ka, 2)
+    D = amq.binary_dots(codes_dev(Wc), codes_dev(Xc), n).cpu().numpy()
+    assert np.array_equal(D, oracle.binary_dots(Wc, Xc, n))                      # bit-exact
+    y = amq.binary_gemm(codes_dev(Wc), dev(Wa, torch.float32), codes_dev(Xc), dev(Xb, torch.float32), n,
+                        bias=dev(bias)).cpu().numpy().astype(np.float64)
+    ref = oracle.binary_gemm(Wc, Wa, Xc, Xb, n, bias.astype(np.float64))
+    assert np.all(np.abs(y - ref) <= parity.output_tolerance(Wa, Xb, n) + 1e-6)
+    # much tighter in practice: fp32 combination of exact integers
+    assert np.abs(y - ref).max() <= 1e-5 * (np.abs(ref).max() + 1)
+    y2 = amq.binary_gemm(codes_dev(Wc), dev(Wa, torch.float32), codes_dev(Xc), dev(Xb, torch.float32), n)
+    assert np.allclose(y2.cpu().numpy(), ref - bias, atol=1e-5 * (np.abs(ref).max() + 1))
+
+
+def test_product_into_strided_output(amq):
+    m, n, batch = 70, 300, 5
+    Wc, Wa = oracle.quantize_rows(synth.normal((m, n), 0.05, 31, 1).astype(np.float64), 2, 2)
+    Xc, Xb = oracle.quantize_rows(synth.uniform((batch, n), -1, 1, 31, 2).astype(np.float64), 2, 2)
+    out = torch.full((batch, 100), 7.0, device="cuda")
+    amq.binary_gemm(codes_dev(Wc), dev(Wa, torch.float32), codes_dev(Xc), dev(Xb, torch.float32), n, y=out[:, :m])
+    ref = oracle.binary_gemm(Wc, Wa, Xc, Xb, n)
+    assert np.allclose(out[:, :m].cpu().numpy(), ref, atol=1e-5)
+    assert torch.all(out[:, m:] == 7.0)          # nothing written past m
+
+
+# ---- cells -----------------------------------------------------------------------------------------------
+
+def cell_setup(cell, I, H, kw, seed, w_std, with_bias=True):
+    gates = 4 if cell == "lstm" else 3
+    W = synth.normal((gates * H, I + H), w_std, seed, 1).astype(np.float64)
+    Wc, Wa = oracle.quantize_rows(W, kw, 2)
+    bias = synth.normal((4 * H,), 0.1, seed, 2) if with_bias else None
+    return Wc, Wa, bias
+
+
+def state_tolerance(Wa, beta, n):
+    # pre-activation tolerance, carried through gates whose slopes are <= 1 (|c| <= a few units)
+    return 3.0 * parity.output_tolerance(Wa, beta, n).max() + 1e-6
+
+
+CELL_CASES = [
+    # cell, I, H, k_w, k_a, batch
+    ("lstm", 300, 300, 2, 2, 1),          # the single-step workload
+    ("lstm", 64, 40, 3, 3, 19),
+    ("lstm", 100, 129, 2, 3, 4),
+    ("gru", 64, 40, 2, 3, 19),
+    ("gru", 100, 129, 3, 2, 5),           # I not a multiple of 32: the column split falls inside a word
+    ("gru", 33, 31, 1, 4, 2),
+]
+
+
+@pytest.mark.parametrize("cell,I,H,kw,ka,batch", CELL_CASES)
+def test_cell_step_matches_oracle(amq, cell, I, H, kw, ka, batch):
+    n = I + H
+    Wc, Wa, bias = cell_setup(cell, I, H, kw, 40 + H, 0.05)
+    x = synth.uniform((batch, I), -1, 1, 41, 1)
+    h = synth.uniform((batch, H), -1, 1, 41, 2)
+    c = synth.uniform((batch, H), -1, 1, 41, 3)
+    ws = amq.new_workspace(I, H, batch, ka)
+    _, beta = oracle.quantize_rows(np.concatenate([x, h], axis=1).astype(np.float64), ka, 2)
+    tol = state_tolerance(Wa, beta, n)
+    dWc, dWa, dbias = codes_dev(Wc), dev(Wa, torch.float32), dev(bias)
+    if cell == "lstm":
+        h_ref, c_ref = oracle.lstm_step(Wc, Wa, bias, I, H, x, h, c, ka, 2)
+        h_out, c_out = amq.lstm_step(dWc, dWa, dbias, I, H, dev(x), dev(h), dev(c), ka, 2, ws)
+        assert np.abs(c_out.cpu().numpy() - c_ref).max() <= tol
+        assert np.abs(h_out.cpu().numpy() - h_ref).max() <= tol
+        h_nb, _ = amq.lstm_step(dWc, dWa, None, I, H, dev(x), dev(h), dev(c), ka, 2, ws)
+        assert np.abs(h_nb.cpu().numpy() - oracle.lstm_step(Wc, Wa, None, I, H, x, h, c, ka, 2)[0]).max() <= tol
+    else:
+        h_ref = oracle.gru_step(Wc, Wa, bias, I, H, x, h, ka, 2)
+        h_out = amq.gru_step(dWc, dWa, dbias, I, H, dev(x), dev(h), ka, 2, ws)
+        assert np.abs(h_out.cpu().numpy() - h_ref).max() <= tol
+    assert amq.workspace_status(ws) == 0
+
+
+@pytest.mark.parametrize("cell,I,H,kw,ka,batch,steps", [("lstm", 48, 32, 2, 2, 1, 6), ("lstm", 40, 24, 3, 3, 7, 5),
+                                                        ("gru", 64, 32, 2, 3, 6, 5)])
+def test_sequence_teacher_forced_and_chained(amq, cell, I, H, kw, ka, batch, steps):
+    n = I + H
+    Wc, Wa, bias = cell_setup(cell, I, H, kw, 50 + H, 0.08)
+    xs = synth.normal((steps, batch, I), 1.0, 51, 1)
+    h0 = np.zeros((batch, H), dtype=np.float32)
+    c0 = np.zeros((batch, H), dtype=np.float32)
+    ws = amq.new_workspace(I, H, batch, ka)
+    dWc, dWa, dbias = codes_dev(Wc), dev(Wa, torch.float32), dev(bias)
+    if cell == "lstm":
+        o_seq, o_last, o_c = oracle.lstm_sequence(Wc, Wa, bias, I, H, xs, h0, c0, ka, 2)
+        g_seq, g_last, g_c = amq.lstm_sequence(dWc, dWa, dbias, I, H, dev(xs), dev(h0), dev(c0), ka, 2, ws,
+                                               want_h_seq=True)
+        _, g_last2, g_c2 = amq.lstm_sequence(dWc, dWa, dbias, I, H, dev(xs), dev(h0), dev(c0), ka, 2, ws)
+        assert torch.equal(g_last, g_last2) and torch.equal(g_c, g_c2) and torch.equal(g_seq[-1], g_last)
+    else:
+        o_seq, o_last = oracle.gru_sequence(Wc, Wa, bias, I, H, xs, h0, ka, 2)
+        g_seq, g_last = amq.gru_sequence(dWc, dWa, dbias, I, H, dev(xs), dev(h0), ka, 2, ws, want_h_seq=True)
+        _, g_last2 = amq.gru_sequence(dWc, dWa, dbias, I, H, dev(xs), dev(h0), ka, 2, ws)
+        assert torch.equal(g_last, g_last2) and torch.equal(g_seq[-1], g_last)
+    # the chained steps of the library reproduce its sequence call bit for bit
+    h, c = dev(h0), dev(c0)
+    for s in range(steps):
+        if cell == "lstm":
+            h, c = amq.lstm_step(dWc, dWa, dbias, I, H, dev(xs[s]), h, c, ka, 2, ws)
+        else:
+            h = amq.gru_step(dWc, dWa, dbias, I, H, dev(xs[s]), h, ka, 2, ws)
+        assert torch.equal(h, g_seq[s])
+    # teacher-forced: every step restarted from the oracle's state must land on the oracle's next state
+    # (reconstructing c_{s-1} for the LSTM by running the oracle step by step)
+    h_prev, c_prev = h0.astype(np.float64), c0.astype(np.float64)
+    for s in range(steps):
+        _, beta = oracle.quantize_rows(np.concatenate([xs[s].astype(np.float64), h_prev], axis=1), ka, 2)
+        tol = state_tolerance(Wa, beta, n)
+        if cell == "lstm":
+            h_ref, c_ref = oracle.lstm_step(Wc, Wa, bias, I, H, xs[s], h_prev, c_prev, ka, 2)
+            h_g, c_g = amq.lstm_step(dWc, dWa, dbias, I, H, dev(xs[s]), dev(h_prev, torch.float32),
+                                     dev(c_prev, torch.float32), ka, 2, ws)
+            assert np.abs(c_g.cpu().numpy() - c_ref).max() <= tol
+            c_prev = c_ref
+        else:
+            h_ref = oracle.gru_step(Wc, Wa, bias, I, H, xs[s], h_prev, ka, 2)
+            h_g = amq.gru_step(dWc, dWa, dbias, I, H, dev(xs[s]), dev(h_prev, torch.float32), ka, 2, ws)
+        assert np.abs(h_g.cpu().numpy() - h_ref).max() <= tol
+        assert np.array_equal(h_ref, o_seq[s])
+        h_prev = h_ref
+    # free-running comparison is reported, not asserted tightly: one flipped activation bit legitimately
+    # moves the trajectory; it must still stay close on these short runs
+    drift = np.abs(g_seq.cpu().numpy() - o_seq).max()
+    print("free-running max |dh| over %d steps: %.3g" % (steps, drift))
+    assert drift <= 0.05
+
+
+def test_sequence_host_variant(amq):
+    I, H, batch, steps, ka = 64, 48, 3, 4, 2
+    Wc, Wa, bias = cell_setup("lstm", I, H, 2, 60, 0.08)
+    xs = torch.from_numpy(synth.normal((steps, batch, I), 1.0, 61, 1)).pin_memory()
+    h0 = torch.zeros((batch, H)).pin_memory()
+    c0 = torch.zeros((batch, H)).pin_memory()
+    ws = amq.new_workspace(I, H, batch, ka)
+    st = amq.new_host_staging(I, H, batch, steps)
+    dWc, dWa, dbias = codes_dev(Wc), dev(Wa, torch.float32), dev(bias)
+    h_last, c_last = torch.empty((batch, H)).pin_memory(), torch.empty((batch, H)).pin_memory()
+    h_seq = torch.empty((steps, batch, H)).pin_memory()
+    amq.lstm_sequence_host(dWc, dWa, dbias, I, H, xs, h0, c0, ka, 2, ws, st, h_last, c_last, h_seq=h_seq)
+    g_seq, g_last, g_c = amq.lstm_sequence(dWc, dWa, dbias, I, H, xs.cuda(), h0.cuda(), c0.cuda(), ka, 2, ws,
+                                           want_h_seq=True)
+    assert torch.equal(h_last, g_last.cpu()) and torch.equal(c_last, g_c.cpu()) and torch.equal(h_seq, g_seq.cpu())
+    G = cell_setup("gru", I, H, 2, 62, 0.08)
+    gh = torch.empty((batch, H)).pin_memory()
+    amq.gru_sequence_host(codes_dev(G[0]), dev(G[1], torch.float32), dev(G[2]), I, H, xs, h0, 3, 2,
+                          amq.new_workspace(I, H, batch, 3), st, gh)
+    _, g2 = amq.gru_sequence(codes_dev(G[0]), dev(G[1], torch.float32), dev(G[2]), I, H, xs.cuda(), h0.cuda(), 3, 2,
+                             amq.new_workspace(I, H, batch, 3))
+    assert torch.equal(gh, g2.cpu())
+
+
+def test_empty_batch_and_zero_steps(amq):
+    I, H, ka = 32, 32, 2
+    Wc, Wa, bias = cell_setup("lstm", I, H, 2, 70, 0.08)
+    ws = amq.new_workspace(I, H, 2, ka)
+    h0 = dev(synth.uniform((2, H), -1, 1, 71, 1))
+    c0 = dev(synth.uniform((2, H), -1, 1, 71, 2))
+    xs = torch.empty((0, 2, I), device="cuda")
+    _, h_last, c_last = amq.lstm_sequence(codes_dev(Wc), dev(Wa, torch.float32), None, I, H, xs, h0, c0, ka, 2, ws)
+    assert torch.equal(h_last, h0) and torch.equal(c_last, c0)
+    codes, coeffs = amq.quantize(torch.empty((0, 64), device="cuda"), 2, 2)
+    assert codes.shape[0] == 0
