@@ -296,9 +296,10 @@ amq_status launch_quantize(const float* src0, int ld0, int n0, const float* src1
 extern "C" amq_status amq_quantize(const float* x, int rows, int n, int ldx, int k, int T,
                                    uint32_t* codes, float* coeffs, void* stream)
 {
-    if (!x || !codes || !coeffs || rows < 0 || n < 1 || ldx < n) return AMQ_ERR_INVALID_ARG;
+    if (rows < 0 || n < 1 || ldx < n) return AMQ_ERR_INVALID_ARG;
     if (!amq::valid_k(k) || T < 0 || n > AMQ_MAX_N) return AMQ_ERR_UNSUPPORTED;
+    if (rows == 0) return AMQ_OK;       // nothing to do; pointers of empty buffers may be NULL
+    if (!x || !codes || !coeffs) return AMQ_ERR_INVALID_ARG;
     if (!amq::aligned16(codes)) return AMQ_ERR_ALIGNMENT;
-    if (rows == 0) return AMQ_OK;
     return amq::launch_quantize(x, ldx, n, nullptr, 0, 0, rows, k, T, codes, coeffs, (cudaStream_t)stream);
 }

@@ -75,6 +75,7 @@ def test_argument_validation_happens_on_the_host(lib):
     assert q(fake, 1, 8193, 8193, 2, 2, fake, fake, None) == -2    # n beyond the maximum
     assert q(fake, 1, 8, 8, 2, 2, odd, fake, None) == -3           # alignment
     assert q(fake, 0, 8, 8, 2, 2, fake, fake, None) == 0           # empty input: nothing to do
+    assert q(None, 0, 8, 8, 2, 2, None, None, None) == 0           # ... even with NULL buffers
     g = lib.amq_binary_gemm
     g.argtypes = [vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, ctypes.c_int, ctypes.c_int, vp, vp,
                   ctypes.c_int, vp]
