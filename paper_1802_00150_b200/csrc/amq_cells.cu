@@ -23,10 +23,28 @@ amq_status validate(const CellCall& c, const void* workspace, size_t workspace_b
     return AMQ_OK;
 }
 
+bool use_persistent(const CellCall& c)
+{
+    int grid, upc;
+    size_t smem;
+    return persistent_supported(c.I, c.H, c.batch, c.k_w, c.k_a, c.gru, &grid, &upc, &smem);
+}
+
+amq_status enqueue_persistent(const CellCall& c, const CellWorkspace& ws, const float* x_seq, int steps,
+                              const float* h0, const float* c0, float* h_seq, float* h_last, float* c_last,
+                              cudaStream_t st)
+{
+    AMQ_CUDA_TRY(cudaMemsetAsync(ws.hx, 0, (size_t)2 * c.H * 8, st));     // stale step tags must not match
+    return launch_rnn_persistent(c.Wcodes, c.Walpha, c.bias, c.I, c.H, c.k_w, c.k_a, c.T, c.gru, x_seq, steps,
+                                 h0, c0, h_seq, h_last, c_last, ws.hx, ws.status, st);
+}
+
 // quantize z = [x ; h_in] into the workspace, then product + gates
 amq_status enqueue_step(const CellCall& c, const CellWorkspace& ws, const float* x, const float* h_in,
                         const float* c_in, float* h_out, float* c_out, cudaStream_t st)
 {
+    if (use_persistent(c))      // batch 1: one launch of the weight-stationary kernel, a sequence of one step
+        return enqueue_persistent(c, ws, x, 1, h_in, c_in, nullptr, h_out, c_out, st);
     amq_status s = launch_quantize(x, c.I, c.I, h_in, c.H, c.H, c.batch, c.k_a, c.T, ws.zcodes, ws.zbeta, st);
     if (s != AMQ_OK) return s;
     GemmArgs a{};
@@ -43,6 +61,8 @@ amq_status enqueue_sequence(const CellCall& c, const CellWorkspace& ws, const fl
 {
     const size_t state_bytes = (size_t)c.batch * c.H * sizeof(float);
     AMQ_CUDA_TRY(cudaMemsetAsync(ws.status, 0, 256, st));
+    if (steps > 0 && use_persistent(c))
+        return enqueue_persistent(c, ws, x_seq, steps, h0, c0, h_seq, h_last, c_last, st);
     if (!c.gru) AMQ_CUDA_TRY(cudaMemcpyAsync(ws.c, c0, state_bytes, cudaMemcpyDeviceToDevice, st));
     const float* h_prev = h0;
     for (int s = 0; s < steps; ++s) {

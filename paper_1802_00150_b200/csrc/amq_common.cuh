@@ -44,6 +44,7 @@ struct CellWorkspace {
     float* zbeta;       // [batch][k_a]
     float* h[2];        // [batch][H] each
     float* c;           // [batch][H]
+    unsigned long long* hx;   // [2][H] exchange words {fp32 bits, step tag} of the persistent kernel
     size_t bytes;
 };
 
@@ -58,6 +59,7 @@ inline CellWorkspace carve_cell_workspace(void* base, int I, int H, int batch, i
     w.h[0] = reinterpret_cast<float*>(p + off);                 off += round_up((size_t)batch * H * 4, 256);
     w.h[1] = reinterpret_cast<float*>(p + off);                 off += round_up((size_t)batch * H * 4, 256);
     w.c = reinterpret_cast<float*>(p + off);                    off += round_up((size_t)batch * H * 4, 256);
+    w.hx = reinterpret_cast<unsigned long long*>(p + off);      off += round_up((size_t)2 * H * 8, 256);
     w.bytes = off;
     return w;
 }
@@ -85,5 +87,14 @@ struct GemmArgs {
 };
 
 amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st);
+
+// Persistent batch-1 recurrent kernel: whether it covers a problem (sizes, shared memory), and its launch.
+bool persistent_supported(int I, int H, int batch, int k_w, int k_a, bool gru, int* grid_out, int* upc_out,
+                          size_t* smem_out);
+amq_status launch_rnn_persistent(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                                 int I, int H, int k_w, int k_a, int T, bool gru,
+                                 const float* x_seq, int steps, const float* h0, const float* c0,
+                                 float* h_seq, float* h_last, float* c_last,
+                                 unsigned long long* hx, uint32_t* status, cudaStream_t st);
 
 }  // namespace amq

@@ -205,6 +205,13 @@ CELL_CASES = [
     ("gru", 64, 40, 2, 3, 19),
     ("gru", 100, 129, 3, 2, 5),           # I not a multiple of 32: the column split falls inside a word
     ("gru", 33, 31, 1, 4, 2),
+    # batch 1 goes through the persistent weight-stationary kernel
+    ("lstm", 1024, 1024, 2, 2, 1),        # the hidden-1024 layer of the benchmark, one step
+    ("lstm", 1536, 1024, 3, 3, 1),        # n = 2560: sixteen elements per thread
+    ("lstm", 100, 77, 1, 4, 1),           # ragged everything
+    ("gru", 128, 96, 2, 3, 1),
+    ("gru", 1024, 600, 3, 2, 1),
+    ("gru", 100, 129, 2, 2, 1),           # I not a multiple of 128: falls back to the two-kernel chain
 ]
 
 
@@ -234,7 +241,8 @@ def test_cell_step_matches_oracle(amq, cell, I, H, kw, ka, batch):
 
 
 @pytest.mark.parametrize("cell,I,H,kw,ka,batch,steps", [("lstm", 48, 32, 2, 2, 1, 6), ("lstm", 40, 24, 3, 3, 7, 5),
-                                                        ("gru", 64, 32, 2, 3, 6, 5)])
+                                                        ("gru", 64, 32, 2, 3, 6, 5), ("gru", 128, 200, 2, 3, 1, 7),
+                                                        ("lstm", 256, 300, 2, 2, 1, 35)])
 def test_sequence_teacher_forced_and_chained(amq, cell, I, H, kw, ka, batch, steps):
     n = I + H
     Wc, Wa, bias = cell_setup(cell, I, H, kw, 50 + H, 0.08)
