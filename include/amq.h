@@ -137,6 +137,32 @@ AMQ_API amq_status amq_lstm_step(const uint32_t* Wcodes, const float* Walpha, co
                          void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * amq_lstm_step for callers that cannot allocate device memory (no counterpart in the paper: this is a
+ * packaging variant of the step above, computing the same thing).  It is meant for code that runs where
+ * cudaMalloc is off limits: inside another application's fixed memory budget, in a loop that must not
+ * enter the driver's allocator once it is running, or after all device memory has been handed out.
+ * The scratch that amq_lstm_step takes as `workspace` (packed codes and coefficients of the quantized
+ * [x ; h_in]) is a fixed array of AMQ_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads
+ * the library holds that much until the process exits.  The call allocates and frees nothing.
+ *   - Arguments as for amq_lstm_step, without the workspace.  A problem whose scratch
+ *     (amq_lstm_step_static_scratch_bytes) exceeds AMQ_STATIC_SCRATCH_BYTES is rejected with
+ *     AMQ_ERR_WORKSPACE before anything is launched.
+ *   - The first call on each device looks up the array's device address (once, with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the last call left.  Each call
+ *     rewrites the part it reads in full before reading it, so nothing needs clearing; but two calls
+ *     whose work overlaps on the GPU (different streams, no ordering) race on it: order them.
+ *   - Always runs the two-kernel chain (row quantizer, then product with the gate epilogue), for every
+ *     batch size.
+ */
+#define AMQ_STATIC_SCRATCH_BYTES (1 << 20)
+AMQ_API size_t amq_lstm_step_static_scratch_bytes(int I, int H, int batch, int k_a);
+AMQ_API amq_status amq_lstm_step_static(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                                int I, int H, int k_w,
+                                const float* x, const float* h_in, const float* c_in, int batch, int k_a, int T,
+                                float* h_out, float* c_out, void* stream);
+
+/*
  * One quantized GRU step.  The paper names the GRU (Sec. 1, Sec. 5) without printing its equations;
  * this library computes the "linear before reset" form:
  *   W: 3H rows in the order r, z, n;  p = W_hat z_hat with z_hat the quantized [x ; h_in];

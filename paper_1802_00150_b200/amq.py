@@ -39,6 +39,8 @@ EXPORTS = {
     "amq_cell_workspace_bytes": (_sz, [_int, _int, _int, _int]),
     "amq_cell_host_staging_bytes": (_sz, [_int, _int, _int, _int]),
     "amq_lstm_step": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _vp, _vp, _int, _int, _int, _vp, _vp, _vp, _sz, _vp]),
+    "amq_lstm_step_static_scratch_bytes": (_sz, [_int, _int, _int, _int]),
+    "amq_lstm_step_static": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _vp, _vp, _int, _int, _int, _vp, _vp, _vp]),
     "amq_gru_step": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _vp, _int, _int, _int, _vp, _vp, _sz, _vp]),
     "amq_lstm_sequence": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _int, _vp, _vp, _int, _int, _int,
                                  _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -184,6 +186,26 @@ def lstm_step(Wcodes, Walpha, bias, I, H, x, h_in, c_in, k_a, T, workspace, h_ou
     c_out = torch.empty_like(c_in) if c_out is None else c_out
     _check(_lib.amq_lstm_step(_ptr(Wcodes), _ptr(Walpha), _ptr(bias), I, H, k_w, _ptr(x), _ptr(h_in), _ptr(c_in),
                               batch, k_a, T, _ptr(h_out), _ptr(c_out), _ptr(workspace), workspace.numel(), _stream()))
+    return h_out, c_out
+
+
+STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def lstm_step_static_scratch_bytes(I, H, batch, k_a):
+    return _lib.amq_lstm_step_static_scratch_bytes(I, H, batch, k_a)
+
+
+def lstm_step_static(Wcodes, Walpha, bias, I, H, x, h_in, c_in, k_a, T, h_out, c_out):
+    """amq_lstm_step without a workspace: the library's built-in scratch array is used, and neither this
+    wrapper nor the call allocates (the caller brings h_out and c_out).  Problems whose scratch exceeds
+    STATIC_SCRATCH_BYTES raise AmqError(-4)."""
+    Wcodes, Walpha = _dev(Wcodes, torch.int32, "Wcodes"), _dev(Walpha, torch.float32, "Walpha")
+    x, h_in, c_in = _dev(x, torch.float32, "x"), _dev(h_in, torch.float32, "h_in"), _dev(c_in, torch.float32, "c_in")
+    h_out, c_out = _dev(h_out, torch.float32, "h_out"), _dev(c_out, torch.float32, "c_out")
+    batch, k_w = h_in.shape[0], Wcodes.shape[1]
+    _check(_lib.amq_lstm_step_static(_ptr(Wcodes), _ptr(Walpha), _ptr(bias), I, H, k_w, _ptr(x), _ptr(h_in),
+                                     _ptr(c_in), batch, k_a, T, _ptr(h_out), _ptr(c_out), _stream()))
     return h_out, c_out
 
 
