@@ -202,6 +202,7 @@ bgemm_popc_kernel(PopcParams p)
 
 amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st)
 {
+    if (gemv_supported(a)) return launch_binary_gemv(a, st);
     PopcParams p;
     p.a = a;
     p.wpr = words_per_row(a.n);

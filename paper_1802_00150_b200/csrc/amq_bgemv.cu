@@ -1,0 +1,212 @@
+// Batch-1 binary matrix-vector product on packed planes (Sec. 4, Fig. 3 left; XOR + bit count,
+// Appendix A): y[r] = sum_i alpha[r][i] * sum_j beta[j] * (n - 2 popcount(W_i[r] xor x_j)) + bias[r].
+//
+// The product streams the packed weight planes from HBM exactly once and is bound by that stream, so
+// the kernel is organised around the loads: a segment of SEG lanes owns one weight row (all k_w planes),
+// lane c of the segment reads the 128-bit chunks c, c + SEG of every plane, and several rows per lane are
+// requested before any is consumed, which keeps enough bytes in flight to cover the DRAM latency.  The k_a
+// activation planes are loop invariant for a lane (it always works on the same columns) and live in
+// registers.
+//
+// Bit counting is the second ceiling right behind the memory one (one POPC per weight word and
+// activation plane issues at a quarter of the logic rate), so pairs of XOR-ed words first go through a
+// carry-save adder on whole words (two LOP3) and only the carries and the final sums are counted.
+#include "amq_common.cuh"
+
+namespace amq {
+
+namespace {
+
+struct GemvParams {
+    const uint4* W;             // [m][k_w][CH] 128-bit chunks
+    const float* Walpha;        // [m][k_w]
+    const uint4* x;             // [k_a][CH]
+    const float* xbeta;         // [k_a]
+    const float* bias;          // [m] or null
+    float* y;                   // EPI_Y
+    int32_t* D;                 // EPI_DOTS: [m][k_w][k_a]
+    int m, n, CH;
+    int epilogue;
+};
+
+// differing bits of (w xor x) over the four words of a chunk, accumulated carry-save:
+// `ones` carries the bit-wise sums, the return value counts the carries (weight 2)
+__device__ __forceinline__ int csa_chunk(const uint4& w, const uint4& x, uint32_t& ones)
+{
+    const uint32_t t0 = w.x ^ x.x, t1 = w.y ^ x.y, t2 = w.z ^ x.z, t3 = w.w ^ x.w;
+    const uint32_t c0 = (ones & t0) | (ones & t1) | (t0 & t1);        // majority -> one LOP3
+    ones ^= t0 ^ t1;
+    const uint32_t c1 = (ones & t2) | (ones & t3) | (t2 & t3);
+    ones ^= t2 ^ t3;
+    return __popc(c0) + __popc(c1);
+}
+
+// sum over the SEG lanes of a segment (exact integers): one warp-wide reduction instruction when the
+// segment is the warp, a shuffle butterfly otherwise
+template <int SEG>
+__device__ __forceinline__ int segment_sum(int v)
+{
+    if (SEG == 32) return __reduce_add_sync(0xffffffffu, v);
+#pragma unroll
+    for (int off = SEG >> 1; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+
+// SEG_LOG2: lanes per row = 1 << SEG_LOG2
+template <int KW, int KA, int CPT, int R, int SEG_LOG2>
+__global__ void __launch_bounds__(256)
+bgemv_kernel(GemvParams p)
+{
+    const int lane = threadIdx.x & 31;
+    constexpr int SEG = 1 << SEG_LOG2;
+    constexpr int spw = 32 >> SEG_LOG2;
+    const int sub = lane & (SEG - 1), seg = lane >> SEG_LOG2;
+    const int CH = p.CH;
+
+    // activation planes of this lane's columns
+    uint4 xr[KA][CPT];
+    bool has[CPT];
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) {
+        has[c] = sub + c * SEG < CH;
+#pragma unroll
+        for (int j = 0; j < KA; ++j)
+            xr[j][c] = has[c] ? __ldg(p.x + (size_t)j * CH + sub + c * SEG) : make_uint4(0, 0, 0, 0);
+    }
+    float beta[KA];
+#pragma unroll
+    for (int j = 0; j < KA; ++j) beta[j] = (p.epilogue == EPI_Y) ? __ldg(p.xbeta + j) : 0.0f;
+
+    const long long rows_per_iter = (long long)spw * R;
+    const long long warp_global = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const long long stride = (long long)gridDim.x * (blockDim.x >> 5) * rows_per_iter;
+
+    for (long long row0 = warp_global * rows_per_iter; row0 < p.m; row0 += stride) {
+        uint4 w[R][KW][CPT];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const long long row = row0 + r * spw + seg;
+            const uint4* src = p.W + (size_t)row * KW * CH + sub;
+#pragma unroll
+            for (int i = 0; i < KW; ++i)
+#pragma unroll
+                for (int c = 0; c < CPT; ++c)
+                    w[r][i][c] = (row < p.m && has[c]) ? __ldcs(src + (size_t)i * CH + c * SEG) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            int P[KW][KA];
+#pragma unroll
+            for (int i = 0; i < KW; ++i)
+#pragma unroll
+                for (int j = 0; j < KA; ++j) {
+                    uint32_t ones = 0;
+                    int carries = 0;
+#pragma unroll
+                    for (int c = 0; c < CPT; ++c) carries += csa_chunk(w[r][i][c], xr[j][c], ones);
+                    P[i][j] = 2 * carries + __popc(ones);
+                }
+            // lanes without a chunk hold w = x = 0 and contribute nothing
+#pragma unroll
+            for (int i = 0; i < KW; ++i)
+#pragma unroll
+                for (int j = 0; j < KA; ++j) P[i][j] = segment_sum<SEG>(P[i][j]);
+            const long long row = row0 + r * spw + seg;
+            if (sub == 0 && row < p.m) {
+                if (p.epilogue == EPI_DOTS) {
+                    int32_t* out = p.D + (size_t)row * KW * KA;
+#pragma unroll
+                    for (int i = 0; i < KW; ++i)
+#pragma unroll
+                        for (int j = 0; j < KA; ++j) out[i * KA + j] = p.n - 2 * P[i][j];
+                } else {
+                    float yv = 0.0f;
+#pragma unroll
+                    for (int i = 0; i < KW; ++i) {
+                        const float al = __ldg(p.Walpha + (size_t)row * KW + i);
+#pragma unroll
+                        for (int j = 0; j < KA; ++j) yv += al * beta[j] * (float)(p.n - 2 * P[i][j]);
+                    }
+                    p.y[row] = yv + (p.bias ? __ldg(p.bias + row) : 0.0f);
+                }
+            }
+        }
+    }
+}
+
+template <int KW, int KA, int CPT, int SEG_LOG2>
+amq_status launch_cfg(const GemvParams& p, cudaStream_t st)
+{
+    constexpr int R = (8 / (KW * CPT)) > 0 ? (8 / (KW * CPT)) : 1;      // about eight 128-bit loads in flight per lane
+    auto kernel = bgemv_kernel<KW, KA, CPT, R, SEG_LOG2>;
+    static thread_local int cached_dev = -1, cached_grid = 0;
+    int dev = 0;
+    AMQ_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != cached_dev) {
+        int sms = 0, per_sm = 0;
+        AMQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        AMQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, 0));
+        cached_grid = sms * (per_sm > 0 ? per_sm : 1);
+        cached_dev = dev;
+    }
+    const long long rows_per_cta = (long long)(32 >> SEG_LOG2) * R * 8;
+    long long need = (p.m + rows_per_cta - 1) / rows_per_cta;
+    const int grid = (int)(need < cached_grid ? need : cached_grid);
+    kernel<<<grid, 256, 0, st>>>(p);
+    AMQ_LAUNCH_CHECK();
+    return AMQ_OK;
+}
+
+// chunks per plane -> lanes per row: 2 (up to 256 columns), 8, 16, 32 with one chunk per lane, 32 with two
+template <int KW, int KA>
+amq_status launch_cpt(const GemvParams& p, cudaStream_t st)
+{
+    if (p.CH <= 2) return launch_cfg<KW, KA, 1, 1>(p, st);
+    if (p.CH <= 8) return launch_cfg<KW, KA, 1, 3>(p, st);
+    if (p.CH <= 16) return launch_cfg<KW, KA, 1, 4>(p, st);
+    if (p.CH <= 32) return launch_cfg<KW, KA, 1, 5>(p, st);
+    return launch_cfg<KW, KA, 2, 5>(p, st);
+}
+
+template <int KW>
+amq_status launch_ka(const GemvParams& p, int k_a, cudaStream_t st)
+{
+    switch (k_a) {
+        case 1: return launch_cpt<KW, 1>(p, st);
+        case 2: return launch_cpt<KW, 2>(p, st);
+        case 3: return launch_cpt<KW, 3>(p, st);
+        case 4: return launch_cpt<KW, 4>(p, st);
+    }
+    return AMQ_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+bool gemv_supported(const GemmArgs& a)
+{
+    return a.batch == 1 && (a.epilogue == EPI_Y || a.epilogue == EPI_DOTS) && words_per_row(a.n) / 4 <= 64;
+}
+
+amq_status launch_binary_gemv(const GemmArgs& a, cudaStream_t st)
+{
+    if (!gemv_supported(a)) return AMQ_ERR_UNSUPPORTED;
+    GemvParams p;
+    p.W = reinterpret_cast<const uint4*>(a.Wcodes);
+    p.Walpha = a.Walpha;
+    p.x = reinterpret_cast<const uint4*>(a.xcodes);
+    p.xbeta = a.xbeta;
+    p.bias = a.bias;
+    p.y = a.y;
+    p.D = a.D;
+    p.m = a.m; p.n = a.n; p.CH = words_per_row(a.n) / 4;
+    p.epilogue = a.epilogue;
+    switch (a.k_w) {
+        case 1: return launch_ka<1>(p, a.k_a, st);
+        case 2: return launch_ka<2>(p, a.k_a, st);
+        case 3: return launch_ka<3>(p, a.k_a, st);
+        case 4: return launch_ka<4>(p, a.k_a, st);
+    }
+    return AMQ_ERR_UNSUPPORTED;
+}
+
+}  // namespace amq

@@ -88,6 +88,10 @@ struct GemmArgs {
 
 amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st);
 
+// Batch-1 streaming kernel (EPI_DOTS / EPI_Y): whether it covers a problem, and its launch.
+bool gemv_supported(const GemmArgs& a);
+amq_status launch_binary_gemv(const GemmArgs& a, cudaStream_t st);
+
 // Persistent batch-1 recurrent kernel: whether it covers a problem (sizes, shared memory), and its launch.
 bool persistent_supported(int I, int H, int batch, int k_w, int k_a, bool gru, int* grid_out, int* upc_out,
                           size_t* smem_out);

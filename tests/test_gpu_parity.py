@@ -149,6 +149,16 @@ GEMM_CASES = [
     (33, 31, 1, 1, 3),
     (257, 300, 1, 4, 17),
     (40, 8192, 2, 2, 2),
+    # batch 1: the streaming matrix-vector kernel (segments of 1..32 lanes per row, one or two chunks per lane)
+    (300, 8192, 3, 3, 1),
+    (1000, 1024, 2, 3, 1),
+    (77, 4100, 4, 4, 1),
+    (513, 100, 1, 2, 1),
+    (64, 6000, 2, 2, 1),
+    (4099, 300, 2, 1, 1),
+    (35, 8192, 4, 4, 1),
+    (9, 1, 3, 2, 1),
+    (21, 9000, 2, 2, 1),                 # beyond 64 chunks per plane: the tiled kernel
 ]
 
 
