@@ -52,23 +52,33 @@ __device__ __forceinline__ int segment_sum(int v)
     return v;
 }
 
-// SEG_LOG2: lanes per row = 1 << SEG_LOG2
-template <int KW, int KA, int CPT, int R, int SEG_LOG2>
+// SEG_LOG2: lanes per row = 1 << SEG_LOG2.  EXACT: every plane has exactly CPT * SEG chunks, so every lane
+// always has work and all load offsets are compile-time constants.
+//
+// A warp works on blocks of 32 consecutive rows.  One pass of the inner loop covers R * (32 / SEG) of them;
+// its loads are issued one pass ahead of the bit counting (register double buffer), so the memory pipe
+// never drains while a warp computes.  After the segment sums every lane of a segment holds the totals of
+// that segment's row; lane `sub` of segment `seg` keeps the ones of row sub * (32 / SEG) + seg, and when
+// the block is complete all 32 lanes fold coefficients and bias and store 32 consecutive outputs at once.
+template <int KW, int KA, int CPT, int R, int SEG_LOG2, bool EXACT>
 __global__ void __launch_bounds__(256)
 bgemv_kernel(GemvParams p)
 {
     const int lane = threadIdx.x & 31;
     constexpr int SEG = 1 << SEG_LOG2;
-    constexpr int spw = 32 >> SEG_LOG2;
+    constexpr int spw = 32 >> SEG_LOG2;            // rows per load instruction of the warp
+    constexpr int PASSES = SEG / R;                // passes per block of 32 rows
+    static_assert(SEG % R == 0, "rows per pass must divide the block");
     const int sub = lane & (SEG - 1), seg = lane >> SEG_LOG2;
-    const int CH = p.CH;
+    const int CH = EXACT ? CPT * SEG : p.CH;
+    const size_t row_chunks = (size_t)KW * CH;
 
     // activation planes of this lane's columns
     uint4 xr[KA][CPT];
     bool has[CPT];
 #pragma unroll
     for (int c = 0; c < CPT; ++c) {
-        has[c] = sub + c * SEG < CH;
+        has[c] = EXACT || (sub + c * SEG < CH);
 #pragma unroll
         for (int j = 0; j < KA; ++j)
             xr[j][c] = has[c] ? __ldg(p.x + (size_t)j * CH + sub + c * SEG) : make_uint4(0, 0, 0, 0);
@@ -77,25 +87,52 @@ bgemv_kernel(GemvParams p)
 #pragma unroll
     for (int j = 0; j < KA; ++j) beta[j] = (p.epilogue == EPI_Y) ? __ldg(p.xbeta + j) : 0.0f;
 
-    const long long rows_per_iter = (long long)spw * R;
+    const long long blocks = ((long long)p.m + 31) >> 5;
     const long long warp_global = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const long long stride = (long long)gridDim.x * (blockDim.x >> 5) * rows_per_iter;
+    const long long total_warps = (long long)gridDim.x * (blockDim.x >> 5);
+    const long long last_row = (long long)p.m - 1;
 
-    for (long long row0 = warp_global * rows_per_iter; row0 < p.m; row0 += stride) {
-        uint4 w[R][KW][CPT];
+    // loads of one pass: rows block * 32 + (pass * R + r) * spw + seg, clamped into the matrix
+    auto load_pass = [&](uint4 (&w)[R][KW][CPT], long long block, int pass) {
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const long long row = row0 + r * spw + seg;
-            const uint4* src = p.W + (size_t)row * KW * CH + sub;
+            long long row = block * 32 + (pass * R + r) * spw + seg;
+            row = row < last_row ? row : last_row;
+            const uint4* src = p.W + (size_t)row * row_chunks + sub;
 #pragma unroll
             for (int i = 0; i < KW; ++i)
 #pragma unroll
-                for (int c = 0; c < CPT; ++c)
-                    w[r][i][c] = (row < p.m && has[c]) ? __ldcs(src + (size_t)i * CH + c * SEG) : make_uint4(0, 0, 0, 0);
+                for (int c = 0; c < CPT; ++c) {
+                    if (EXACT) w[r][i][c] = __ldcs(src + (i * CPT + c) * SEG);
+                    else w[r][i][c] = has[c] ? __ldcs(src + (size_t)i * CH + c * SEG) : make_uint4(0, 0, 0, 0);
+                }
+        }
+    };
+
+    int mine[KW][KA];           // totals of this lane's row of the current block
+#pragma unroll
+    for (int i = 0; i < KW; ++i)
+#pragma unroll
+        for (int j = 0; j < KA; ++j) mine[i][j] = 0;
+
+    // the passes of all blocks, in order, are dealt out to the warps in equal contiguous shares (a share
+    // may begin and end inside a block; each warp then finishes only the rows of the passes it ran)
+    const long long total = blocks * PASSES;
+    const long long share = total / total_warps, extra = total % total_warps;
+    long long g = warp_global * share + (warp_global < extra ? warp_global : extra);
+    const long long g_end = g + share + (warp_global < extra ? 1 : 0);
+    int first_pass = (int)(g % PASSES);          // first pass this warp ran in the current block
+
+    auto step = [&](uint4 (&cur)[R][KW][CPT], uint4 (&nxt)[R][KW][CPT]) {
+        const long long block = g / PASSES;
+        const int pass = (int)(g - block * PASSES);
+        if (g + 1 < g_end) {
+            const long long nblock = (g + 1) / PASSES;
+            load_pass(nxt, nblock, (int)(g + 1 - nblock * PASSES));
         }
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            int P[KW][KA];
+            const bool keep = sub == pass * R + r;
 #pragma unroll
             for (int i = 0; i < KW; ++i)
 #pragma unroll
@@ -103,55 +140,74 @@ bgemv_kernel(GemvParams p)
                     uint32_t ones = 0;
                     int carries = 0;
 #pragma unroll
-                    for (int c = 0; c < CPT; ++c) carries += csa_chunk(w[r][i][c], xr[j][c], ones);
-                    P[i][j] = 2 * carries + __popc(ones);
+                    for (int c = 0; c < CPT; ++c) carries += csa_chunk(cur[r][i][c], xr[j][c], ones);
+                    // lanes without a chunk hold w = x = 0 and contribute nothing
+                    const int sum = segment_sum<SEG>(2 * carries + __popc(ones));
+                    if (keep) mine[i][j] = sum;
                 }
-            // lanes without a chunk hold w = x = 0 and contribute nothing
-#pragma unroll
-            for (int i = 0; i < KW; ++i)
-#pragma unroll
-                for (int j = 0; j < KA; ++j) P[i][j] = segment_sum<SEG>(P[i][j]);
-            const long long row = row0 + r * spw + seg;
-            if (sub == 0 && row < p.m) {
+        }
+        if (pass == PASSES - 1 || g + 1 == g_end) {
+            const long long row = block * 32 + sub * spw + seg;       // this lane's row of the block
+            const int my_pass = sub / R;
+            if (row < p.m && my_pass >= first_pass && my_pass <= pass) {
                 if (p.epilogue == EPI_DOTS) {
                     int32_t* out = p.D + (size_t)row * KW * KA;
 #pragma unroll
                     for (int i = 0; i < KW; ++i)
 #pragma unroll
-                        for (int j = 0; j < KA; ++j) out[i * KA + j] = p.n - 2 * P[i][j];
+                        for (int j = 0; j < KA; ++j) out[i * KA + j] = p.n - 2 * mine[i][j];
                 } else {
                     float yv = 0.0f;
 #pragma unroll
                     for (int i = 0; i < KW; ++i) {
                         const float al = __ldg(p.Walpha + (size_t)row * KW + i);
 #pragma unroll
-                        for (int j = 0; j < KA; ++j) yv += al * beta[j] * (float)(p.n - 2 * P[i][j]);
+                        for (int j = 0; j < KA; ++j) yv += al * beta[j] * (float)(p.n - 2 * mine[i][j]);
                     }
                     p.y[row] = yv + (p.bias ? __ldg(p.bias + row) : 0.0f);
                 }
             }
+            first_pass = 0;
         }
+        ++g;
+    };
+
+    uint4 wa[R][KW][CPT], wb[R][KW][CPT];
+    if (g < g_end) load_pass(wa, g / PASSES, (int)(g % PASSES));
+    while (g < g_end) {
+        step(wa, wb);
+        if (!(g < g_end)) break;
+        step(wb, wa);
     }
 }
 
 template <int KW, int KA, int CPT, int SEG_LOG2>
 amq_status launch_cfg(const GemvParams& p, cudaStream_t st)
 {
-    constexpr int R = (8 / (KW * CPT)) > 0 ? (8 / (KW * CPT)) : 1;      // about eight 128-bit loads in flight per lane
-    auto kernel = bgemv_kernel<KW, KA, CPT, R, SEG_LOG2>;
-    static thread_local int cached_dev = -1, cached_grid = 0;
+    constexpr int SEG = 1 << SEG_LOG2;
+    constexpr int R0 = (8 / (KW * CPT)) > 0 ? (8 / (KW * CPT)) : 1;     // about eight 128-bit loads per lane and pass
+    constexpr int R = R0 < SEG ? R0 : SEG;
+    const bool exact = p.CH == CPT * SEG;
+    auto kernel = exact ? bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, true> : bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, false>;
+    static thread_local int cached_dev = -1, cached_grid[2] = {0, 0};
     int dev = 0;
     AMQ_CUDA_TRY(cudaGetDevice(&dev));
     if (dev != cached_dev) {
-        int sms = 0, per_sm = 0;
+        int sms = 0;
         AMQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        AMQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, 256, 0));
-        cached_grid = sms * (per_sm > 0 ? per_sm : 1);
+        for (int e = 0; e < 2; ++e) {
+            int per_sm = 0;
+            if (e) AMQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, true>, 256, 0));
+            else AMQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, false>, 256, 0));
+            cached_grid[e] = sms * (per_sm > 0 ? per_sm : 1);
+        }
         cached_dev = dev;
     }
-    const long long rows_per_cta = (long long)(32 >> SEG_LOG2) * R * 8;
-    long long need = (p.m + rows_per_cta - 1) / rows_per_cta;
-    const int grid = (int)(need < cached_grid ? need : cached_grid);
+    constexpr int PASSES = SEG / R;
+    const long long passes = ((long long)p.m + 31) / 32 * PASSES;
+    const long long need = (passes + 31) / 32;                          // at least four passes per warp
+    const int limit = cached_grid[exact ? 1 : 0];
+    const int grid = (int)(need < limit ? need : limit);
     kernel<<<grid, 256, 0, st>>>(p);
     AMQ_LAUNCH_CHECK();
     return AMQ_OK;
