@@ -116,6 +116,14 @@ AMQ_API amq_status amq_binary_gemm(const uint32_t* Wcodes, const float* Walpha, 
                            const uint32_t* xcodes, const float* xbeta, int batch, int k_a,
                            const float* bias, float* y, int ldy, void* stream);
 
+/*
+ * Synchronises `stream`, then reads and clears the library's device-side status word of the current
+ * device: AMQ_OK, or AMQ_ERR_TIMEOUT if a bounded wait inside a product kernel ran out since the last
+ * read (the outputs of that call are then undefined).  Covers amq_binary_dots, amq_binary_gemm and the
+ * product inside the cell calls; the sequence kernels report through amq_workspace_status as well.
+ */
+AMQ_API amq_status amq_device_status(void* stream);
+
 /* Scratch for the cell calls below (steps and sequences), in bytes; 0 on invalid arguments. */
 AMQ_API size_t amq_cell_workspace_bytes(int I, int H, int batch, int k_a);
 /* Additional device staging needed by the *_host variants (x_seq, states and results), in bytes. */

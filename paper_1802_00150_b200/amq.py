@@ -36,6 +36,7 @@ EXPORTS = {
     "amq_unpack": (_int, [_vp, _vp, _int, _int, _int, _vp, _vp]),
     "amq_binary_dots": (_int, [_vp, _int, _int, _int, _vp, _int, _int, _vp, _vp]),
     "amq_binary_gemm": (_int, [_vp, _vp, _int, _int, _int, _vp, _vp, _int, _int, _vp, _vp, _int, _vp]),
+    "amq_device_status": (_int, [_vp]),
     "amq_cell_workspace_bytes": (_sz, [_int, _int, _int, _int]),
     "amq_cell_host_staging_bytes": (_sz, [_int, _int, _int, _int]),
     "amq_lstm_step": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _vp, _vp, _int, _int, _int, _vp, _vp, _vp, _sz, _vp]),
@@ -160,6 +161,11 @@ def binary_gemm(Wcodes, Walpha, xcodes, xbeta, n, bias=None, y=None):
     _check(_lib.amq_binary_gemm(_ptr(Wcodes), _ptr(Walpha), m, n, k_w, _ptr(xcodes), _ptr(xbeta), batch, k_a,
                                 _ptr(bias), _ptr(y), y.stride(0) if batch > 1 else max(m, y.stride(0)), _stream()))
     return y
+
+
+def device_status():
+    """0, or -6 when a bounded device-side wait of a product kernel ran out since the last call."""
+    return _lib.amq_device_status(_stream())
 
 
 def cell_workspace_bytes(I, H, batch, k_a):

@@ -203,6 +203,7 @@ bgemm_popc_kernel(PopcParams p)
 amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st)
 {
     if (gemv_supported(a)) return launch_binary_gemv(a, st);
+    if (gemm_tc_supported(a)) return launch_binary_gemm_tc(a, st);
     PopcParams p;
     p.a = a;
     p.wpr = words_per_row(a.n);
@@ -256,6 +257,14 @@ amq_status amq_binary_gemm(const uint32_t* Wcodes, const float* Walpha, int m, i
     a.xcodes = xcodes; a.xbeta = xbeta; a.batch = batch; a.k_a = k_a;
     a.bias = bias; a.epilogue = amq::EPI_Y; a.y = y; a.ldy = ldy;
     return amq::launch_binary_gemm(a, (cudaStream_t)stream);
+}
+
+amq_status amq_device_status(void* stream)
+{
+    uint32_t word = 0;
+    amq_status s = amq::read_tc_status((cudaStream_t)stream, &word);
+    if (s != AMQ_OK) return s;
+    return word == 0 ? AMQ_OK : AMQ_ERR_TIMEOUT;
 }
 
 }  // extern "C"

@@ -92,6 +92,12 @@ amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st);
 bool gemv_supported(const GemmArgs& a);
 amq_status launch_binary_gemv(const GemmArgs& a, cudaStream_t st);
 
+// Tensor-core kernel (tcgen05, batch >= 16): whether it covers a problem, its launch, and its status word
+// (nonzero after a bounded device-side wait ran out; cleared by the read).
+bool gemm_tc_supported(const GemmArgs& a);
+amq_status launch_binary_gemm_tc(const GemmArgs& a, cudaStream_t st);
+amq_status read_tc_status(cudaStream_t st, uint32_t* out);
+
 // Persistent batch-1 recurrent kernel: whether it covers a problem (sizes, shared memory), and its launch.
 bool persistent_supported(int I, int H, int batch, int k_w, int k_a, bool gru, int* grid_out, int* upc_out,
                           size_t* smem_out);
