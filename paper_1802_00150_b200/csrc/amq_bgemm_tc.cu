@@ -8,28 +8,37 @@
 // The planes stay bit-packed in global memory.  A CTA expands the bits of its tile into signed bytes in
 // shared memory: bit 1 -> -64, bit 0 -> +64 on both operands, so a byte product is 4096 * (+-1 * +-1) and a
 // 32-bit accumulator holds 4096 * (dot of the +-1 vectors); pad positions (0 in both operands) add one
-// each and are subtracted again.  Expanding costs one shift and one logic operation per four bytes:
-// output register s of a 32-bit word keeps bits s, s + 8, s + 16, s + 24 in its four bytes, i.e. the K
-// positions inside a word are permuted, identically for both operands, which a dot product does not see.
+// each and are subtracted again.  Expanding costs one shift (issued as a multiplication, on the FMA pipe)
+// and one three-input logic operation per four bytes: output register s of a 32-bit word keeps bits s,
+// s + 8, s + 16, s + 24 in its four bytes, i.e. the K positions inside a word are permuted, identically for
+// both operands, which a dot product does not see.  What bounds the expansion is the shared-memory store
+// bandwidth (128 operand bytes per row and stage), not the arithmetic.
 //
-// Shared-memory operand layout: K-major, no swizzle, 8-row x 16-byte core matrices, stored as
-// [16-byte K chunk][group of 8 rows][row][16 bytes]; one MMA instruction consumes K = 32 bytes = the two
-// chunks of one packed word.  Expansion of K stage s + 1 (all threads, generic-proxy stores, then a
-// proxy fence) overlaps the asynchronous MMAs of stage s; an mbarrier per buffer, signalled by
-// tcgen05.commit, says when a buffer may be overwritten.  Every wait is bounded: when one runs out the CTA
-// records the failure in a status word, skips its stores, frees its tensor memory and returns.
+// Shared-memory operand layout: K-major with the 128-byte swizzle: a pipeline stage holds 128 bytes of K per
+// operand row, rows are 128 bytes apart, groups of 8 rows 1024 bytes apart, and the 16-byte chunk j of row r
+// sits at chunk position j xor (r mod 8).  One MMA instruction consumes K = 32 bytes = the two chunks of one
+// packed word; its descriptor start address advances by 32 bytes per word inside the swizzled row.
+//
+// Roles: expander threads, one per operand row (plane-rows of the weight tile, then rows of the activation
+// tile), turn packed words into operand bytes, stage by stage (128 bit positions of K per stage, three or
+// four stages in flight); where the thread budget allows, two such groups take the stages in turn, so that
+// the serial latency of one stage (wait, expand, proxy fence, arrive) is overlapped; one more warp issues
+// the MMAs.  A "full" mbarrier per stage is signalled by every expander thread of the group (generic-proxy
+// stores, proxy fence, arrive), an "empty" one by tcgen05.commit when the MMAs that read the stage have
+// completed.  A CTA may own two M tiles that share one expanded activation tile, which halves the
+// expansion work per MMA.  Every wait is bounded: when one runs out the CTA records the failure in a status
+// word, skips its stores, frees its tensor memory and returns.
 #include "amq_common.cuh"
 
 namespace amq {
 
 namespace {
 
-constexpr int TC_THREADS = 256;
-constexpr int TILE_M = 128;                 // stacked weight plane-rows per CTA (= TMEM lanes)
-constexpr int STAGE_WORDS = 8;              // packed words of K per pipeline stage (256 bit positions)
-constexpr int A_LBO = TILE_M / 8 * 128;     // bytes between 16-byte K chunks of the A tile
-constexpr int A_STAGE_BYTES = STAGE_WORDS * 2 * A_LBO;
-constexpr unsigned WAIT_LIMIT = 1u << 22;   // polls of an mbarrier before giving up
+constexpr int MAX_THREADS = 1024;           // expander threads (one or two per operand row) plus the warp that issues the MMAs
+constexpr int TILE_M = 128;                 // stacked weight plane-rows per M tile (= TMEM lanes)
+constexpr int STAGE_WORDS = 4;              // packed words of K per pipeline stage (128 bit positions)
+constexpr int MAX_STAGES = 4;
+constexpr unsigned WAIT_LIMIT = 1u << 20;   // attempts on an mbarrier before giving up
 
 __device__ uint32_t g_tc_status;            // nonzero after a bounded wait ran out (sticky until read)
 
@@ -37,12 +46,20 @@ struct TcParams {
     GemmArgs a;
     int gates;      // 1 plain, 4 LSTM, 3 GRU
     int units;      // plain: m; cells: H
-    int UT;         // units per tile
+    int UT;         // units per M tile
+    int MT;         // M tiles per CTA (1 or 2)
     int TB;         // batch entries per tile (multiple of 16)
     int nseg;       // 1, or 2 for the GRU (columns [0,I) and [I,n))
     int wpr;
     int n_mma;      // TB * k_a: N of the MMA, multiple of 16, <= 256
-    int tmem_cols;  // power of two >= nseg * n_mma
+    int tmem_cols;  // power of two >= MT * nseg * n_mma
+    int nstages;    // pipeline depth
+    int expanders;  // operand rows of a stage, MT * 128 + n_mma, rounded up to whole warps
+    int groups;     // expander groups (1 or 2) that take the pipeline steps in turn, `expanders` threads each
+    // run-time copies of compile-time constants: the shifts of the expansion as multipliers (so that they
+    // issue on the FMA pipe) and its two byte masks (so that one LOP3 takes both from registers)
+    uint32_t mul[8];
+    uint32_t mask_sign, mask_half;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -63,7 +80,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return done != 0;
 }
 
-// bounded wait; false when it ran out
+// bounded wait of the single MMA-issuing thread; false when it ran out
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
     for (unsigned i = 0; i < WAIT_LIMIT; ++i)
@@ -71,11 +88,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     return false;
 }
 
-// K-major, no swizzle: start address, leading (K chunk) byte offset, stride (8-row group) byte offset
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
+// the same for the many expander threads: between attempts the thread sleeps, so that waiters do not take
+// issue slots from the warps that have work
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity)
 {
-    return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)((lbo >> 4) & 0x3fffu) << 16) |
-           ((uint64_t)((sbo >> 4) & 0x3fffu) << 32) | (1ull << 46);
+    if (mbar_try_wait(bar, parity)) return true;
+    for (unsigned i = 0; i < WAIT_LIMIT; ++i) {
+        __nanosleep(40);
+        if (mbar_try_wait(bar, parity)) return true;
+    }
+    return false;
+}
+
+// K-major, 128-byte swizzle: start address (the tile base is 1024-byte aligned), leading byte offset unused (1),
+// stride byte offset = 1024 bytes between groups of 8 rows, descriptor version 1, layout type 2
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
+{
+    return (uint64_t)((addr >> 4) & 0x3fffu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
 __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
@@ -101,49 +130,62 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16])
         : "r"(taddr) : "memory");
 }
 
-// 128 packed bits of one plane-row -> 128 signed bytes (-64 for bit 1, +64 for bit 0), written as eight
-// 16-byte K chunks `lbo` bytes apart starting at `dst`
-__device__ __forceinline__ void expand_store(const uint4& v, unsigned char* dst, int lbo)
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w)
 {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        uint32_t y[8];
-#pragma unroll
-        for (int s = 0; s < 8; ++s) y[s] = ((w[q] << (7 - s)) & 0x80808080u) ^ 0x40404040u;
-        *reinterpret_cast<uint4*>(dst + (2 * q) * lbo) = make_uint4(y[0], y[1], y[2], y[3]);
-        *reinterpret_cast<uint4*>(dst + (2 * q + 1) * lbo) = make_uint4(y[4], y[5], y[6], y[7]);
-    }
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" :: "r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+
+// (x & a) ^ b in one three-input logic instruction
+__device__ __forceinline__ uint32_t and_xor(uint32_t x, uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(x), "r"(a), "r"(b));
+    return d;
+}
+
+// exact conversion of a small integer (|v| < 2^22) on the FMA pipe instead of the conversion unit
+__device__ __forceinline__ float small_int_to_float(int v)
+{
+    return __int_as_float(v + 0x4B400000) - 12582912.0f;
 }
 
 __device__ __forceinline__ float logistic(float v) { return 1.0f / (1.0f + __expf(-v)); }
 
 template <int KA>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(MAX_THREADS, 1)
 bgemm_tc_kernel(TcParams p)
 {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const GemmArgs& a = p.a;
     const int k_w = a.k_w;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int TM = p.UT * p.gates;                  // weight rows of the tile
-    const int TMp = TM * k_w;                       // plane-rows in use (<= 128)
+    const int TM = p.UT * p.gates;                  // weight rows of an M tile
+    const int TMp = TM * k_w;                       // plane-rows in use per M tile (<= 128)
+    const int MT = p.MT, S = p.nstages, G = p.groups;
+    const int EXP = p.expanders;                    // operand rows rounded up to whole warps
+    const int mma_warp = (G * EXP) >> 5, nthreads = G * EXP + 32;
     const int n_mma = p.n_mma;
-    const int b_lbo = n_mma * 16;                   // bytes between K chunks of the B tile
-    const int stage_bytes = A_STAGE_BYTES + STAGE_WORDS * 2 * b_lbo;
-    const int u0 = blockIdx.x * p.UT, b0 = blockIdx.y * p.TB;
+    const int a_stage_bytes = MT * TILE_M * 128;    // 128 bytes of K per row and stage
+    const int stage_bytes = a_stage_bytes + n_mma * 128;
+    const int u0 = blockIdx.x * p.UT * MT, b0 = blockIdx.y * p.TB;
 
     unsigned char* stage_base = smem_raw;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + 2 * stage_bytes);      // [2] buffer-free barriers
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)S * stage_bytes);   // [S]
+    uint64_t* empty_bar = full_bar + MAX_STAGES;                                            // [S]
+    uint64_t* done_bar = empty_bar + MAX_STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done_bar + 1);
+    volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     if (tid == 0) {
-        mbar_init(smem_u32(&bars[0]), 1);
-        mbar_init(smem_u32(&bars[1]), 1);
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), (uint32_t)EXP);
+            mbar_init(smem_u32(&empty_bar[s]), 1);
+        }
+        mbar_init(smem_u32(done_bar), 1);
+        *failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncwarp();
-    if (warp == 0) {
+    if (warp == mma_warp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -153,187 +195,234 @@ bgemm_tc_kernel(TcParams p)
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
 
-    // ---- expansion roles: per stage a thread expands one 128-bit chunk of an A row and two of a B row ----
-    const int a_row = tid & (TILE_M - 1), a_half = tid >> 7;        // A: row, which of the two chunks of the stage
-    const uint32_t* a_src = nullptr;
-    if (a_row < TMp) {
-        const int l = a_row / k_w, i = a_row - l * k_w;
-        const int u = u0 + l / p.gates, gate = l % p.gates;
-        if (u < p.units) a_src = a.Wcodes + (((size_t)gate * p.units + u) * k_w + i) * p.wpr;
-    }
-    const uint32_t* b_src = nullptr;                                // B: row tid (stacked activation plane)
-    if (tid < n_mma) {
-        const int b = b0 + tid / KA, j = tid % KA;
-        if (b < a.batch) b_src = a.xcodes + ((size_t)b * KA + j) * p.wpr;
-    }
-    const int a_off = (a_row >> 3) * 128 + (a_row & 7) * 16;
-    const int b_off = (tid >> 3) * 128 + (tid & 7) * 16;
-
-    const int CH = p.wpr >> 2;                                      // 128-bit chunks along K
-    const int stages = (CH + 1) >> 1;
+    const int CH = p.wpr >> 2;                                      // 128-bit chunks along K = pipeline steps
     const int split_word = (p.nseg == 2) ? (a.I >> 5) : p.wpr;      // first word of the second column segment
-    const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
 
-    auto load_a = [&](int s) -> uint4 {
-        const int c = 2 * s + a_half;
-        return (a_src && c < CH) ? __ldg(reinterpret_cast<const uint4*>(a_src) + c) : make_uint4(0, 0, 0, 0);
-    };
-    auto load_b = [&](int s, int h) -> uint4 {
-        const int c = 2 * s + h;
-        return (b_src && c < CH) ? __ldg(reinterpret_cast<const uint4*>(b_src) + c) : make_uint4(0, 0, 0, 0);
-    };
-
-    uint4 va = load_a(0), vb0 = load_b(0, 0), vb1 = load_b(0, 1);
-    bool ok = true;
-    for (int s = 0; s < stages; ++s) {
-        const int buf = s & 1;
-        unsigned char* sa = stage_base + buf * stage_bytes;
-        unsigned char* sb = sa + A_STAGE_BYTES;
-        // the MMAs that read this buffer two stages ago must have completed
-        if (s >= 2) ok = mbar_wait(smem_u32(&bars[buf]), (uint32_t)(((s >> 1) + 1) & 1));
-        if (__syncthreads_or(!ok)) { ok = false; break; }          // uniform: every thread leaves the loop
-
-        const uint4 ca = va, cb0 = vb0, cb1 = vb1;
-        if (s + 1 < stages) { va = load_a(s + 1); vb0 = load_b(s + 1, 0); vb1 = load_b(s + 1, 1); }
-        expand_store(ca, sa + a_off + (a_half * 8) * A_LBO, A_LBO);
-        if (tid < n_mma) {
-            expand_store(cb0, sb + b_off, b_lbo);
-            expand_store(cb1, sb + b_off + 8 * b_lbo, b_lbo);
+    if (warp < mma_warp) {
+        // ---- expanders: G groups of EXP threads take the steps in turn; inside a group thread r owns operand
+        //      row r (A plane-rows first, then the B rows) ----
+        const int grp = tid / EXP, r_all = tid - grp * EXP;
+        const uint4* src = nullptr;
+        uint32_t dst0;                                              // shared address of the row in stage 0
+        if (r_all < MT * TILE_M) {
+            const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
+            if (r < TMp) {
+                const int l = r / k_w, i = r - l * k_w;
+                const int u = u0 + mt * p.UT + l / p.gates, gate = l % p.gates;
+                if (u < p.units)
+                    src = reinterpret_cast<const uint4*>(a.Wcodes + (((size_t)gate * p.units + u) * k_w + i) * p.wpr);
+            }
+            dst0 = smem_u32(stage_base) + r_all * 128;
+        } else {
+            const int r = r_all - MT * TILE_M;
+            const int b = b0 + r / KA, j = r % KA;
+            if (r < n_mma && b < a.batch) src = reinterpret_cast<const uint4*>(a.xcodes + ((size_t)b * KA + j) * p.wpr);
+            dst0 = smem_u32(stage_base) + a_stage_bytes + r * 128;
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic-proxy stores -> async proxy
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-        if (tid == 0) {
+        const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
+        uint32_t off[8];                                            // swizzled position of chunk j: j xor (row mod 8)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) off[j] = (uint32_t)((j ^ (r_all & 7)) << 4);
+        uint32_t mul[7];
+#pragma unroll
+        for (int s = 0; s < 7; ++s) mul[s] = p.mul[s];
+        const uint32_t m_sign = p.mask_sign, m_half = p.mask_half;  // 0x80808080, 0x40404040
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+
+        uint4 cur = (src && grp < CH) ? __ldg(src + grp) : zero;    // own steps: grp, grp + G, ..
+        uint4 nxt = (src && grp + G < CH) ? __ldg(src + grp + G) : zero;
+        int buf = grp;                                              // G <= S
+        uint32_t empty_parity = 1;                                  // parity that means "never used" on the first lap
+        for (int c = grp; c < CH; c += G) {
+            const uint4 v = cur;
+            cur = nxt;
+            nxt = (src && c + 2 * G < CH) ? __ldg(src + c + 2 * G) : zero;
+            // the MMAs that read this buffer one lap ago must have completed
+            if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; break; }
+            if (writes) {
+                const uint32_t base = dst0 + (uint32_t)(buf * stage_bytes);
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t y[8];
+#pragma unroll
+                    for (int s = 0; s < 7; ++s) y[s] = and_xor(w[q] * mul[s], m_sign, m_half);     // w << (7 - s)
+                    y[7] = and_xor(w[q], m_sign, m_half);
+                    st_shared_v4(base + off[2 * q], y[0], y[1], y[2], y[3]);
+                    st_shared_v4(base + off[2 * q + 1], y[4], y[5], y[6], y[7]);
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
+            buf += G;
+            if (buf >= S) { buf -= S; empty_parity ^= 1u; }
+        }
+    } else if (lane == 0) {
+        // ---- MMA issuer ----
+        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+        const uint64_t desc_base = smem_desc(smem_u32(stage_base)); // descriptor of stage 0, tile 0, word 0
+        int buf = 0;
+        uint32_t full_parity = 0;
+        for (int c = 0; c < CH; ++c) {
+            if (!mbar_wait(smem_u32(&full_bar[buf]), full_parity)) { *failed = 1; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t sa_addr = smem_u32(sa), sb_addr = smem_u32(sb);
-            for (int q = 0; q < STAGE_WORDS; ++q) {
-                const int word = s * STAGE_WORDS + q;
-                if (word >= p.wpr) break;
+            // descriptors of the stage: start addresses are below 256 KiB, so adding to the low word never carries
+            const uint64_t adesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
+            const uint64_t bdesc0 = adesc0 + (uint64_t)(a_stage_bytes >> 4);
+#pragma unroll
+            for (int qq = 0; qq < STAGE_WORDS; ++qq) {
+                const int word = c * STAGE_WORDS + qq;
                 const int seg = word >= split_word ? 1 : 0;
                 const uint32_t accumulate = (word != 0 && word != split_word) ? 1u : 0u;
-                mma_i8(tmem_base + seg * n_mma,
-                       smem_desc(sa_addr + q * 2 * A_LBO, A_LBO, 128),
-                       smem_desc(sb_addr + q * 2 * b_lbo, b_lbo, 128), idesc, accumulate);
+                mma_i8(tmem_base + seg * n_mma, adesc0 + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                if (MT == 2)
+                    mma_i8(tmem_base + (p.nseg + seg) * n_mma, adesc0 + (TILE_M * 128 >> 4) + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
             }
-            mma_commit(smem_u32(&bars[buf]));
+            mma_commit(smem_u32(&empty_bar[buf]));
+            if (++buf == S) { buf = 0; full_parity ^= 1u; }
         }
+        if (!*failed) mma_commit(smem_u32(done_bar));               // covers every MMA issued above
     }
-    // all MMAs done: the commit of the last stage covers every earlier one
-    if (ok) {
-        const int last = stages - 1;
-        ok = mbar_wait(smem_u32(&bars[last & 1]), (uint32_t)((last >> 1) & 1));
-    }
+    __syncwarp();
+
+    // all MMAs done?
+    bool ok = !*failed;
+    if (ok) ok = mbar_wait_relaxed(smem_u32(done_bar), 0);
     if (__syncthreads_or(!ok)) {
         // give the tensor core time to drain what was issued, then release tensor memory and leave
         if (tid == 0) atomicExch(&g_tc_status, 1u);
         __nanosleep(1000000);
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncthreads();
-        if (warp == 0)
+        if (warp == mma_warp)
             asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
         return;
     }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
     // ---- epilogue 1: tensor memory -> registers -> partial products in shared memory ----
-    // thread = plane-row (lane of tensor memory); warps 0-3 take the lower half of the batch entries of the
-    // tile, warps 4-7 the upper half, 16 entries (16 * KA columns) at a time
-    float* Yt = reinterpret_cast<float*>(smem_raw);                 // [nseg][128][TB + 1], reuses the stage buffers
+    // thread = plane-row (lane of tensor memory); warp w reads lane quarter w & 3; with eight or more warps the
+    // batch entries of the tile are split between warps 0-3 and 4-7.  Columns arrive 16 at a time; entry e
+    // of a block of 16 entries owns columns e * KA .. e * KA + KA - 1 of its 16 * KA columns.
+    float* Yt = reinterpret_cast<float*>(smem_raw);                 // [MT][nseg][128][TB + 1], reuses the stage buffers
+    float* sBeta = Yt + (size_t)MT * p.nseg * TILE_M * (p.TB + 1);  // [TB][KA]
     const int ldy = p.TB + 1;
-    const int pr = (warp & 3) * 32 + lane;
-    const int pad = p.wpr * 32 - a.n;                               // pad positions, all in the last segment
-    {
-        const int l = pr / k_w, i = pr - l * k_w;
-        const int u = u0 + l / p.gates, gate = l % p.gates;
-        const bool row_ok = pr < TMp && u < p.units;
-        const size_t row = (size_t)gate * p.units + u;
-        const float alpha = (row_ok && a.epilogue != EPI_DOTS) ? __ldg(a.Walpha + row * k_w + i) : 0.0f;
-        const int groups = p.TB >> 4, half = (groups + 1) >> 1;
+    for (int idx = tid; idx < p.TB * KA; idx += nthreads) {
+        const int b = b0 + idx / KA;
+        sBeta[idx] = (b < a.batch && a.epilogue != EPI_DOTS) ? __ldg(a.xbeta + (size_t)b * KA + idx % KA) : 0.0f;
+    }
+    __syncthreads();
+    const int epi_halves = (mma_warp >= 8) ? 2 : 1;
+    if (warp < 4 * epi_halves) {
+        const int pr = (warp & 3) * 32 + lane;
+        const int pad = p.wpr * 32 - a.n;                           // pad positions, all in the last segment
+        const int groups = p.TB >> 4, half = (epi_halves == 2) ? (groups + 1) >> 1 : groups;
         const int g_lo = (warp < 4) ? 0 : half, g_hi = (warp < 4) ? half : groups;
-        for (int seg = 0; seg < p.nseg; ++seg) {
-            const int corr = (seg == p.nseg - 1) ? pad : 0;
-            const int len = (p.nseg == 2) ? (seg == 0 ? a.I : a.n - a.I) : a.n;
-            (void)len;
-            for (int g = g_lo; g < g_hi; ++g) {
-                int acc[KA][16];
-#pragma unroll
-                for (int c = 0; c < KA; ++c)
-                    tmem_ld16(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(seg * n_mma + (g * KA + c) * 16), acc[c]);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const int bb = g * 16 + e, b = b0 + bb;
+        for (int mt = 0; mt < MT; ++mt) {
+            const int l = pr / k_w, i = pr - l * k_w;
+            const int u = u0 + mt * p.UT + l / p.gates, gate = l % p.gates;
+            const bool row_ok = pr < TMp && u < p.units;
+            const size_t row = (size_t)gate * p.units + u;
+            const float alpha = (row_ok && a.epilogue != EPI_DOTS) ? __ldg(a.Walpha + row * k_w + i) : 0.0f;
+            for (int seg = 0; seg < p.nseg; ++seg) {
+                const int corr = (seg == p.nseg - 1) ? pad : 0;
+                float* yrow = Yt + ((size_t)(mt * p.nseg + seg) * TILE_M + pr) * ldy;
+                const uint32_t tbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((mt * p.nseg + seg) * n_mma);
+                for (int g = g_lo; g < g_hi; ++g) {
                     float y = 0.0f;
 #pragma unroll
-                    for (int j = 0; j < KA; ++j) {
-                        const int col = e * KA + j;                  // compile-time position inside the group
-                        const int D = (acc[col >> 4][col & 15] >> 12) - corr;
-                        if (a.epilogue == EPI_DOTS) {
-                            if (row_ok && b < a.batch)
-                                a.D[(((size_t)b * a.m + row) * k_w + i) * KA + j] = D;
-                        } else {
-                            const float be = (b < a.batch) ? __ldg(a.xbeta + (size_t)b * KA + j) : 0.0f;
-                            y += be * (float)D;
+                    for (int c = 0; c < KA; ++c) {
+                        int acc[16];
+                        tmem_ld16(tbase + (uint32_t)((g * KA + c) * 16), acc);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            const int col = c * 16 + k, e = col / KA, j = col % KA;      // compile-time
+                            const int bb = g * 16 + e;
+                            const int D = (acc[k] >> 12) - corr;
+                            if (a.epilogue == EPI_DOTS) {
+                                const int b = b0 + bb;
+                                if (row_ok && b < a.batch) a.D[(((size_t)b * a.m + row) * k_w + i) * KA + j] = D;
+                            } else {
+                                y += sBeta[bb * KA + j] * small_int_to_float(D);
+                                if (j == KA - 1) { yrow[bb] = alpha * y; y = 0.0f; }
+                            }
                         }
                     }
-                    if (a.epilogue != EPI_DOTS) Yt[((size_t)seg * TILE_M + pr) * ldy + bb] = alpha * y;
                 }
             }
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 0)
+    if (warp == mma_warp)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
     if (a.epilogue == EPI_DOTS) return;
 
     // ---- epilogue 2: sum the k_w planes of each weight row, bias, gates ----
+    // thread -> (row or unit, every `bstep`-th batch entry): one division per thread, none per output
     const int TB = p.TB;
-    auto pre = [&](int seg, int l, int bb) -> float {
-        float s = 0.0f;
-        for (int i = 0; i < k_w; ++i) s += Yt[((size_t)seg * TILE_M + l * k_w + i) * ldy + bb];
-        return s;
-    };
-    if (a.epilogue == EPI_Y) {
-        for (int idx = tid; idx < TM * TB; idx += TC_THREADS) {
-            const int bb = idx / TM, l = idx - bb * TM;              // consecutive threads -> consecutive rows
-            const int row = u0 + l, b = b0 + bb;
-            if (row < a.m && b < a.batch)
-                a.y[(size_t)b * a.ldy + row] = pre(0, l, bb) + (a.bias ? __ldg(a.bias + row) : 0.0f);
-        }
-    } else if (a.epilogue == EPI_LSTM) {
-        const int H = a.H;
-        for (int idx = tid; idx < p.UT * TB; idx += TC_THREADS) {
-            const int bb = idx / p.UT, ul = idx - bb * p.UT;
-            const int u = u0 + ul, b = b0 + bb;
-            if (u < H && b < a.batch) {
+    const int per_tile = (a.epilogue == EPI_Y) ? TM : p.UT;         // rows (plain) or units (cells) of an M tile
+    const int items = MT * per_tile;
+    const int lanes_b = nthreads / items;                           // threads sharing one row / unit (0: fewer threads than items)
+    const int bsub = lanes_b > 0 ? tid / items : 0;
+    const int bstep = lanes_b > 0 ? lanes_b : 1;
+    const int istep = lanes_b > 0 ? items : nthreads;
+    if (lanes_b > 0 && bsub >= lanes_b) return;
+    for (int item = lanes_b > 0 ? tid - bsub * items : tid; item < items; item += istep) {
+        const int mt = item / per_tile, li = item - mt * per_tile;
+        if (a.epilogue == EPI_Y) {
+            const int row = u0 + item;
+            if (row >= a.m) continue;
+            const float bias = a.bias ? __ldg(a.bias + row) : 0.0f;
+            const float* y0 = Yt + ((size_t)(mt * p.nseg) * TILE_M + li * k_w) * ldy;
+            for (int bb = bsub; bb < TB && b0 + bb < a.batch; bb += bstep) {
+                float s = bias;
+                for (int i = 0; i < k_w; ++i) s += y0[i * ldy + bb];
+                a.y[(size_t)(b0 + bb) * a.ldy + row] = s;
+            }
+        } else if (a.epilogue == EPI_LSTM) {
+            const int H = a.H, u = u0 + item;
+            if (u >= H) continue;
+            float bias4[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) bias4[g] = a.bias ? __ldg(a.bias + g * H + u) : 0.0f;
+            const float* y0 = Yt + ((size_t)(mt * p.nseg) * TILE_M + li * 4 * k_w) * ldy;
+            for (int bb = bsub; bb < TB && b0 + bb < a.batch; bb += bstep) {
                 float g4[4];
 #pragma unroll
-                for (int g = 0; g < 4; ++g) g4[g] = pre(0, ul * 4 + g, bb) + (a.bias ? __ldg(a.bias + g * H + u) : 0.0f);
+                for (int g = 0; g < 4; ++g) {
+                    float s = bias4[g];
+                    for (int i = 0; i < k_w; ++i) s += y0[(g * k_w + i) * ldy + bb];
+                    g4[g] = s;
+                }
                 const float ig = logistic(g4[0]), fg = logistic(g4[1]), og = logistic(g4[2]);
                 const float gg = tanhf(g4[3]);
-                const size_t o = (size_t)b * H + u;
+                const size_t o = (size_t)(b0 + bb) * H + u;
                 const float c = fg * a.c_in[o] + ig * gg;
                 a.c_out[o] = c;
                 a.h_out[o] = og * tanhf(c);
             }
-        }
-    } else {    // EPI_GRU
-        const int H = a.H;
-        for (int idx = tid; idx < p.UT * TB; idx += TC_THREADS) {
-            const int bb = idx / p.UT, ul = idx - bb * p.UT;
-            const int u = u0 + ul, b = b0 + bb;
-            if (u < H && b < a.batch) {
+        } else {    // EPI_GRU
+            const int H = a.H, u = u0 + item;
+            if (u >= H) continue;
+            const float br = a.bias ? __ldg(a.bias + u) : 0.0f, bz = a.bias ? __ldg(a.bias + H + u) : 0.0f;
+            const float bnx = a.bias ? __ldg(a.bias + 2 * H + u) : 0.0f;
+            const float bnh = a.bias ? __ldg(a.bias + 3 * H + u) : 0.0f;
+            const float* yx = Yt + ((size_t)(mt * 2 + 0) * TILE_M + li * 3 * k_w) * ldy;
+            const float* yh = Yt + ((size_t)(mt * 2 + 1) * TILE_M + li * 3 * k_w) * ldy;
+            for (int bb = bsub; bb < TB && b0 + bb < a.batch; bb += bstep) {
                 float px[3], ph[3];
 #pragma unroll
-                for (int g = 0; g < 3; ++g) { px[g] = pre(0, ul * 3 + g, bb); ph[g] = pre(1, ul * 3 + g, bb); }
-                const float br = a.bias ? __ldg(a.bias + u) : 0.0f, bz = a.bias ? __ldg(a.bias + H + u) : 0.0f;
-                const float bnx = a.bias ? __ldg(a.bias + 2 * H + u) : 0.0f;
-                const float bnh = a.bias ? __ldg(a.bias + 3 * H + u) : 0.0f;
+                for (int g = 0; g < 3; ++g) {
+                    float sx = 0.0f, sh = 0.0f;
+                    for (int i = 0; i < k_w; ++i) { sx += yx[(g * k_w + i) * ldy + bb]; sh += yh[(g * k_w + i) * ldy + bb]; }
+                    px[g] = sx; ph[g] = sh;
+                }
                 const float rg = logistic(px[0] + ph[0] + br);
                 const float zg = logistic(px[1] + ph[1] + bz);
                 const float cand = tanhf(px[2] + bnx + rg * (ph[2] + bnh));
-                const size_t o = (size_t)b * H + u;
+                const size_t o = (size_t)(b0 + bb) * H + u;
                 a.h_out[o] = (1.0f - zg) * cand + zg * a.h_in[o];
             }
         }
@@ -359,21 +448,35 @@ bool plan(const GemmArgs& a, TcPlan* out)
     } else { p.gates = 1; p.units = a.m; }
     p.UT = TILE_M / (p.gates * a.k_w);
     if (p.UT < 1) return false;
-    // batch entries per tile: multiples of 16, N = TB * k_a <= 256 (and both accumulators of the GRU in 512 columns)
+    // batch entries per tile: multiples of 16, N = TB * k_a <= 256
     int tb_max = (256 / a.k_a) / 16 * 16;
     if (tb_max > 128) tb_max = 128;
-    const int tiles = (a.batch + tb_max - 1) / tb_max;
-    p.TB = ((a.batch + tiles - 1) / tiles + 15) / 16 * 16;
+    const int ntiles = (a.batch + tb_max - 1) / tb_max;
+    p.TB = ((a.batch + ntiles - 1) / ntiles + 15) / 16 * 16;
     p.n_mma = p.TB * a.k_a;
+    // two M tiles per CTA when their accumulators fit tensor memory and enough CTAs remain to fill the GPU
+    const int mtiles = (p.units + p.UT - 1) / p.UT;
+    const int btiles = (a.batch + p.TB - 1) / p.TB;
+    p.MT = (2 * p.nseg * p.n_mma <= 512 && (long long)(mtiles / 2) * btiles >= 2 * 148) ? 2 : 1;
     int cols = 32;
-    while (cols < p.nseg * p.n_mma) cols <<= 1;
+    while (cols < p.MT * p.nseg * p.n_mma) cols <<= 1;
     if (cols > 512) return false;
     p.tmem_cols = cols;
-    const size_t stage = (size_t)A_STAGE_BYTES + (size_t)STAGE_WORDS * 2 * p.n_mma * 16;
-    if ((size_t)p.nseg * TILE_M * (p.TB + 1) * 4 > 2 * stage) return false;
+    const size_t stage = (size_t)128 * (p.MT * TILE_M + p.n_mma);
+    const size_t epi = ((size_t)p.MT * p.nseg * TILE_M * (p.TB + 1) + (size_t)p.TB * a.k_a) * 4;
+    int S = (int)((220 * 1024) / stage);
+    if (S > MAX_STAGES) S = MAX_STAGES;
+    if (S < 2) return false;
+    if (epi > S * stage) return false;
+    p.nstages = S;
+    p.expanders = (p.MT * TILE_M + p.n_mma + 31) / 32 * 32;
+    p.groups = (2 * p.expanders + 32 <= MAX_THREADS) ? 2 : 1;
+    for (int sft = 0; sft < 8; ++sft) p.mul[sft] = 1u << (7 - sft);
+    p.mask_sign = 0x80808080u;
+    p.mask_half = 0x40404040u;
     out->p = p;
-    out->smem = 2 * stage + 64;
-    out->grid = dim3((unsigned)((p.units + p.UT - 1) / p.UT), (unsigned)((a.batch + p.TB - 1) / p.TB));
+    out->smem = S * stage + (2 * MAX_STAGES + 1) * 8 + 16;
+    out->grid = dim3((unsigned)((mtiles + p.MT - 1) / p.MT), (unsigned)btiles);
     return out->grid.y <= 65535u && out->smem <= 227 * 1024;
 }
 
@@ -382,7 +485,7 @@ amq_status launch_ka(const TcPlan& pl, cudaStream_t st)
 {
     auto kernel = bgemm_tc_kernel<KA>;
     AMQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
-    kernel<<<pl.grid, TC_THREADS, pl.smem, st>>>(pl.p);
+    kernel<<<pl.grid, pl.p.groups * pl.p.expanders + 32, pl.smem, st>>>(pl.p);
     AMQ_LAUNCH_CHECK();
     return AMQ_OK;
 }
