@@ -301,9 +301,8 @@ bgemm_tc_kernel(TcParams p)
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
     // ---- epilogue 1: tensor memory -> registers -> partial products in shared memory ----
-    // thread = plane-row (lane of tensor memory); warp w reads lane quarter w & 3; with eight or more warps the
-    // batch entries of the tile are split between warps 0-3 and 4-7.  Columns arrive 16 at a time; entry e
-    // of a block of 16 entries owns columns e * KA .. e * KA + KA - 1 of its 16 * KA columns.
+    // thread = plane-row (lane of tensor memory).  Columns arrive 16 at a time; entry e of a block of 16
+    // batch entries owns columns e * KA .. e * KA + KA - 1 of the block's 16 * KA columns.
     float* Yt = reinterpret_cast<float*>(smem_raw);                 // [MT][nseg][128][TB + 1], reuses the stage buffers
     float* sBeta = Yt + (size_t)MT * p.nseg * TILE_M * (p.TB + 1);  // [TB][KA]
     const int ldy = p.TB + 1;
@@ -312,42 +311,44 @@ bgemm_tc_kernel(TcParams p)
         sBeta[idx] = (b < a.batch && a.epilogue != EPI_DOTS) ? __ldg(a.xbeta + (size_t)b * KA + idx % KA) : 0.0f;
     }
     __syncthreads();
-    const int epi_halves = (mma_warp >= 8) ? 2 : 1;
-    if (warp < 4 * epi_halves) {
+    // every group of four warps covers the 128 lanes once (warp w reads lane quarter w & 3); the work items
+    // (M tile, column segment, block of 16 batch entries) are dealt out to those groups in turn
+    const int epi_slots = mma_warp >> 2;                            // whole groups of four warps among the expanders
+    if (warp < 4 * epi_slots) {
         const int pr = (warp & 3) * 32 + lane;
+        const int slot = warp >> 2;
         const int pad = p.wpr * 32 - a.n;                           // pad positions, all in the last segment
-        const int groups = p.TB >> 4, half = (epi_halves == 2) ? (groups + 1) >> 1 : groups;
-        const int g_lo = (warp < 4) ? 0 : half, g_hi = (warp < 4) ? half : groups;
-        for (int mt = 0; mt < MT; ++mt) {
-            const int l = pr / k_w, i = pr - l * k_w;
-            const int u = u0 + mt * p.UT + l / p.gates, gate = l % p.gates;
+        const int groups = p.TB >> 4;
+        const int l = pr / k_w, i = pr - l * k_w;
+        const int gate = l % p.gates;
+        const int items1 = MT * p.nseg * groups;
+        for (int item = slot; item < items1; item += epi_slots) {
+            const int g = item % groups, ms = item / groups;        // ms = mt * nseg + seg
+            const int mt = ms / p.nseg, seg = ms - mt * p.nseg;
+            const int u = u0 + mt * p.UT + l / p.gates;
             const bool row_ok = pr < TMp && u < p.units;
             const size_t row = (size_t)gate * p.units + u;
             const float alpha = (row_ok && a.epilogue != EPI_DOTS) ? __ldg(a.Walpha + row * k_w + i) : 0.0f;
-            for (int seg = 0; seg < p.nseg; ++seg) {
-                const int corr = (seg == p.nseg - 1) ? pad : 0;
-                float* yrow = Yt + ((size_t)(mt * p.nseg + seg) * TILE_M + pr) * ldy;
-                const uint32_t tbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((mt * p.nseg + seg) * n_mma);
-                for (int g = g_lo; g < g_hi; ++g) {
-                    float y = 0.0f;
+            const int corr = (seg == p.nseg - 1) ? pad : 0;
+            float* yrow = Yt + ((size_t)ms * TILE_M + pr) * ldy;
+            const uint32_t tbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(ms * n_mma);
+            float y = 0.0f;
 #pragma unroll
-                    for (int c = 0; c < KA; ++c) {
-                        int acc[16];
-                        tmem_ld16(tbase + (uint32_t)((g * KA + c) * 16), acc);
-                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            for (int c = 0; c < KA; ++c) {
+                int acc[16];
+                tmem_ld16(tbase + (uint32_t)((g * KA + c) * 16), acc);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const int col = c * 16 + k, e = col / KA, j = col % KA;      // compile-time
-                            const int bb = g * 16 + e;
-                            const int D = (acc[k] >> 12) - corr;
-                            if (a.epilogue == EPI_DOTS) {
-                                const int b = b0 + bb;
-                                if (row_ok && b < a.batch) a.D[(((size_t)b * a.m + row) * k_w + i) * KA + j] = D;
-                            } else {
-                                y += sBeta[bb * KA + j] * small_int_to_float(D);
-                                if (j == KA - 1) { yrow[bb] = alpha * y; y = 0.0f; }
-                            }
-                        }
+                for (int k = 0; k < 16; ++k) {
+                    const int col = c * 16 + k, e = col / KA, j = col % KA;      // compile-time
+                    const int bb = g * 16 + e;
+                    const int D = (acc[k] >> 12) - corr;
+                    if (a.epilogue == EPI_DOTS) {
+                        const int b = b0 + bb;
+                        if (row_ok && b < a.batch) a.D[(((size_t)b * a.m + row) * k_w + i) * KA + j] = D;
+                    } else {
+                        y += sBeta[bb * KA + j] * small_int_to_float(D);
+                        if (j == KA - 1) { yrow[bb] = alpha * y; y = 0.0f; }
                     }
                 }
             }
@@ -376,7 +377,17 @@ bgemm_tc_kernel(TcParams p)
             if (row >= a.m) continue;
             const float bias = a.bias ? __ldg(a.bias + row) : 0.0f;
             const float* y0 = Yt + ((size_t)(mt * p.nseg) * TILE_M + li * k_w) * ldy;
-            for (int bb = bsub; bb < TB && b0 + bb < a.batch; bb += bstep) {
+            const int bend = (a.batch - b0 < TB) ? a.batch - b0 : TB;
+            int bb = bsub;
+            for (; bb + 3 * bstep < bend; bb += 4 * bstep) {       // four entries in flight
+                float s[4] = {bias, bias, bias, bias};
+                for (int i = 0; i < k_w; ++i)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) s[q] += y0[i * ldy + bb + q * bstep];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) a.y[(size_t)(b0 + bb + q * bstep) * a.ldy + row] = s[q];
+            }
+            for (; bb < bend; bb += bstep) {
                 float s = bias;
                 for (int i = 0; i < k_w; ++i) s += y0[i * ldy + bb];
                 a.y[(size_t)(b0 + bb) * a.ldy + row] = s;
