@@ -44,7 +44,7 @@ def parse_args():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-extras", action="store_true", help="skip the cold-GEMV bandwidth line")
+    ap.add_argument("--no-extras", action="store_true", help="skip the cold-GEMV bandwidth lines and the batched-regime lines")
     return ap.parse_args()
 
 
@@ -380,6 +380,8 @@ def run_ours(args, wl):
         }
         if not args.no_extras and world == 1:
             line["gemv_cold"] = cold_gemv(amq, torch, dev, flush, peak, peak_kind)
+            line["batched"] = batched_lines(amq, torch, dev, flush, peak, peak_kind)
+            assert amq.device_status() == 0
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(wl, unit)
     if dist is not None:
@@ -389,35 +391,99 @@ def run_ours(args, wl):
         print(json.dumps(line))
 
 
-def cold_gemv(amq, torch, dev, flush, peak, peak_kind):
-    """Batch-1 binary GEMV on packed planes far larger than L2 (HBM-bound): achieved GB/s of packed weights."""
-    m, n, k_w, k_a = 131072, 8192, 2, 2
-    wpr = amq.words_per_row(n)
-    g = torch.Generator(device=dev)
-    g.manual_seed(0)
-    Wcodes = torch.randint(-2 ** 31, 2 ** 31 - 1, (m, k_w, wpr), dtype=torch.int32, device=dev, generator=g)
-    Walpha = torch.rand((m, k_w), device=dev, generator=g) * 0.02
-    x = torch.from_numpy(synth.uniform((1, n), -1, 1, 0, 9)).to(dev)
-    xc, xb = amq.quantize(x, k_a, 2)
-    y = torch.empty((1, m), device=dev)
-    for _ in range(3):
-        amq.binary_gemm(Wcodes, Walpha, xc, xb, n, y=y)
+def _event_ms(torch, fn, flush, iters):
+    """Median device time of fn (one launch chain) with the L2 flushed, untimed, before every run."""
     times = []
-    for i in range(10):
-        flush.fill_(i)
+    for i in range(iters):
+        flush.fill_(i & 0xFF)
         s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s.record()
-        amq.binary_gemm(Wcodes, Walpha, xc, xb, n, y=y)
+        fn()
         e.record()
         torch.cuda.synchronize()
         times.append(s.elapsed_time(e))
-    ms = float(np.median(times))
-    alg = Wcodes.numel() * 4 + Walpha.numel() * 4 + m * 4 + xc.numel() * 4
-    gbs = alg / (ms * 1e-3) / 1e9
-    return {"workload": "batch-1 binary GEMV %dx%d, k_w=%d, k_a=%d, packed planes %d MiB (random bits), cold" % (
-                m, n, k_w, k_a, Wcodes.numel() * 4 >> 20),
-            "ms": ms, "achieved": gbs, "unit": "GB/s", "peak": peak, "frac": gbs / peak, "peak_kind": "of " + peak_kind,
-            "frac_of_nominal_8000": gbs / 8000.0, "algorithmic_bytes": int(alg)}
+    return float(np.median(times))
+
+
+def _burst_ms(torch, fn, iters):
+    """Device time per call over `iters` calls enqueued back to back (for kernels shorter than a launch)."""
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record()
+    for _ in range(iters):
+        fn()
+    e.record()
+    torch.cuda.synchronize()
+    return s.elapsed_time(e) / iters
+
+
+def cold_gemv(amq, torch, dev, flush, peak, peak_kind):
+    """Batch-1 binary GEMV on packed planes far larger than L2 (HBM-bound): achieved GB/s of packed weights."""
+    out = []
+    for m, n, k_w, k_a in ((131072, 8192, 2, 2), (262144, 8192, 2, 2), (131072, 8192, 3, 3), (1048576, 1024, 2, 2)):
+        wpr = amq.words_per_row(n)
+        g = torch.Generator(device=dev)
+        g.manual_seed(0)
+        Wcodes = torch.randint(-2 ** 31, 2 ** 31 - 1, (m, k_w, wpr), dtype=torch.int32, device=dev, generator=g)
+        Walpha = torch.rand((m, k_w), device=dev, generator=g) * 0.02
+        x = torch.from_numpy(synth.uniform((1, n), -1, 1, 0, 9)).to(dev)
+        xc, xb = amq.quantize(x, k_a, 2)
+        y = torch.empty((1, m), device=dev)
+        for _ in range(3):
+            amq.binary_gemm(Wcodes, Walpha, xc, xb, n, y=y)
+        ms = _event_ms(torch, lambda: amq.binary_gemm(Wcodes, Walpha, xc, xb, n, y=y), flush, 10)
+        alg = Wcodes.numel() * 4 + Walpha.numel() * 4 + m * 4 + xc.numel() * 4
+        gbs = alg / (ms * 1e-3) / 1e9
+        out.append({"workload": "batch-1 binary GEMV %dx%d, k_w=%d, k_a=%d, packed planes %d MiB (random bits), cold" % (
+                        m, n, k_w, k_a, Wcodes.numel() * 4 >> 20),
+                    "ms": ms, "bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": peak, "frac": gbs / peak,
+                    "peak_kind": "of " + peak_kind, "frac_of_nominal_8000": gbs / 8000.0, "algorithmic_bytes": int(alg)})
+        del Wcodes, Walpha, y
+    return out
+
+
+def batched_lines(amq, torch, dev, flush, hbm_peak, peak_kind):
+    """The batched (binary GEMM) regime and the bulk quantizer, one line per benchmark shape.  The tensor-core
+    product is held against the int8 peak = 2 x the measured dense bf16 figure (nominal int8 : bf16 ratio)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        bf16 = float(json.load(open(path))["bf16_tflops"])
+        tkind = "of measured bf16 x 2"
+    except Exception:
+        bf16, tkind = 1590.0, "of fallback bf16 x 2"
+    int8_tops = 2.0 * bf16
+    out = []
+    for name in ("lstm1024_b64", "gru2048_b256", "proj32768_b512"):
+        wl = synth.WORKLOADS[name]
+        wpr = amq.words_per_row(wl.n)
+        g = torch.Generator(device=dev)
+        g.manual_seed(1)
+        W = torch.randn((wl.m, wl.n), device=dev, generator=g) * wl.w_std
+        Wcodes, Walpha = amq.quantize(W, wl.k_w, wl.T)
+        acts = torch.randn((wl.batch, wl.n), device=dev, generator=g)
+        xc, xb = amq.quantize(acts, wl.k_a, wl.T)
+        y = torch.empty((wl.batch, wl.m), device=dev)
+        ms = _burst_ms(torch, lambda: amq.binary_gemm(Wcodes, Walpha, xc, xb, wl.n, y=y), 20)
+        mac = wl.m * wl.k_w * wl.batch * wl.k_a * wpr * 32
+        tops = 2.0 * mac / (ms * 1e-3) / 1e12
+        out.append({"workload": "binary GEMM of %s: stacked M=%d, N=%d, K=%d bit positions" % (
+                        name, wl.m * wl.k_w, wl.batch * wl.k_a, wpr * 32),
+                    "ms": ms, "bound": "tensor", "achieved": tops, "unit": "TOP/s (int8, 2 per bit-MAC)", "peak": int8_tops,
+                    "frac": tops / int8_tops, "peak_kind": tkind, "bit_mac_per_s": mac / (ms * 1e-3)})
+        msq = _burst_ms(torch, lambda: amq.quantize(acts, wl.k_a, wl.T, codes=xc, coeffs=xb), 20)
+        out.append({"workload": "on-line quantizer of %s: %d vectors of %d, k=%d, T=%d" % (name, wl.batch, wl.n, wl.k_a, wl.T),
+                    "ms": msq, "bound": "latency"})
+        if name == "proj32768_b512":
+            msb = _event_ms(torch, lambda: amq.quantize(W, wl.k_w, wl.T, codes=Wcodes, coeffs=Walpha), flush, 10)
+            alg = W.numel() * 4 + Wcodes.numel() * 4 + Walpha.numel() * 4
+            gbs = alg / (msb * 1e-3) / 1e9
+            out.append({"workload": "bulk row-wise quantization %dx%d, k=%d, T=%d, cold" % (wl.m, wl.n, wl.k_w, wl.T),
+                        "ms": msb, "bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": hbm_peak, "frac": gbs / hbm_peak,
+                        "peak_kind": "of " + peak_kind, "algorithmic_bytes": int(alg)})
+        del W, Wcodes, Walpha, acts, xc, xb, y
+    return out
 
 
 def cpu_baseline(wl, unit):
