@@ -228,6 +228,28 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+# ---- replicas: what differs between ranks, and how their measurements are combined ----------------------
+
+def rank_workload(wl, rank):
+    """Every rank runs its own sequences (seed offset by rank) through the same model (weights are not offset)."""
+    return synth.scaled(wl, seed=wl.seed + 1000 * rank) if rank else wl
+
+
+def combine_over_ranks(dist, device, total_ms, e2e_total_ms, launches):
+    """Slowest rank's times (MAX) and the launches of all ranks (SUM); no data-path collective exists."""
+    import torch
+    t = torch.tensor([total_ms, e2e_total_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    lt = torch.tensor([launches], device=device, dtype=torch.int64)
+    dist.all_reduce(lt, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), int(lt[0])
+
+
+def whole_job_value(world, units, steps, total_ms):
+    """Units all ranks processed / the slowest rank's time."""
+    return world * units * steps / (total_ms * 1e-3)
+
+
 # ---- our arm ---------------------------------------------------------------------------------------------
 
 def run_ours(args, wl):
@@ -247,7 +269,7 @@ def run_ours(args, wl):
     stream = torch.cuda.current_stream()
 
     # inputs: every rank draws its own sequences (seed offset by rank); weights are the same model
-    wl_rank = synth.scaled(wl, seed=wl.seed + 1000 * rank) if rank else wl
+    wl_rank = rank_workload(wl, rank)
     ins = synth.inputs(wl_rank)
     W = torch.from_numpy(synth.weights(wl)).to(dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)        # 256 MiB > L2 (126 MB)
@@ -338,18 +360,13 @@ def run_ours(args, wl):
     e2e_total_ms = float(sum(ms_e2e))
     e2e_iters = len(ms_e2e)
     if dist is not None:
-        t = torch.tensor([total_ms, e2e_total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_total_ms = float(t[0]), float(t[1])
-        lt = torch.tensor([launches], device=dev, dtype=torch.int64)
-        dist.all_reduce(lt, op=dist.ReduceOp.SUM)
-        launches = int(lt[0])
+        total_ms, e2e_total_ms, launches = combine_over_ranks(dist, dev, total_ms, e2e_total_ms, launches)
     assert amq.workspace_status(ws) == 0 if wl.cell != "proj" else True
 
     units = units_per_step(wl)
     unit = "timesteps/s" if wl.cell != "proj" else "passes/s"
-    value = world * units * args.steps / (total_ms * 1e-3)
-    e2e_value = world * units * e2e_iters / (e2e_total_ms * 1e-3)
+    value = whole_job_value(world, units, args.steps, total_ms)
+    e2e_value = whole_job_value(world, units, e2e_iters, e2e_total_ms)
     peak, peak_kind = measured_peaks()
 
     line = None
