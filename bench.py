@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by workload; the summaries are under profiles/.  None = not captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"lstm1024_b1": 2331904 + 8192}     # rnn_persistent_kernel, profiles/rnn_persistent_kernel_lstm1024_b1.txt
 
 
 def parse_args():
@@ -377,7 +377,8 @@ def run_ours(args, wl):
             kernel_name = "bulk quantize + binary GEMM (whole step)"
         else:
             alg_bytes = algorithmic_bytes_per_timestep(wl) * wl.steps
-            kernel_name = "sequence step chain (quantize + binary product with gate epilogue)"
+            kernel_name = ("rnn_persistent_kernel (one launch = the whole sequence)" if wl.batch == 1
+                           else "chain of quantize_kernel + bgemm_tc_kernel per timestep")
         achieved = alg_bytes / (step_ms * 1e-3) / 1e9
         line = {
             "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
