@@ -1,11 +1,20 @@
 // Device-side body of the alternating multi-bit quantizer (Algorithm 2), shared by the stand-alone
 // row quantizer kernel and by the persistent recurrent kernel, which quantizes [x ; h] in place.
 //
-// A "group" of threads owns one vector; thread g of a group of G threads holds elements j*G + g,
-// j < EPT, in registers.  Data-parallel form of Algorithm 1 ("maintaining a mask vector ... operate BST
-// for all entries simultaneously", Sec. 3): the 2^k - 1 midpoints of the ascending level table are
-// non-decreasing, so the leaf the tree descent reaches is the number of midpoints that are <= w; every
-// element counts them with branch-free compares and looks its sign pattern up in a packed code table.
+// A "group" of threads owns one vector; every thread holds EPT of its elements in registers (which ones is
+// the caller's choice).  Data-parallel form of Algorithm 1 ("maintaining a mask vector ... operate BST for
+// all entries simultaneously", Sec. 3): every element descends the tree over the 2^k - 1 midpoints of the
+// ascending level table with k compares and predicated selects of the next midpoint (no branches), and the
+// leaf index looks the sign pattern up in one small bit table per plane.
+//
+// Instruction economy of the inner loops (they decide the throughput of bulk quantization): inputs are
+// canonicalised (-0.0 -> +0.0), after which "r >= 0" is exactly "sign bit clear" for every residue the
+// greedy step can produce, so a sign plane is gathered with one funnel shift per element, a residue is
+// updated as r - copysign(alpha, r) with one logic operation and one add, and +-w for the refit sums is one
+// logic operation; the refit sums of a cycle are accumulated in the same pass that assigns the codes.
+// Elements past the end of the vector are zeros that take part in every loop unmasked: their bits are
+// cleared at the end, they add nothing to B^T w, the Gram matrix is counted on masked words, and their known
+// contribution to the greedy |r| sums (all of them follow the trajectory of a zero element) is subtracted.
 //
 // Arithmetic: sums over the vector are fp32 (per thread, then a fixed butterfly / warp order, so results
 // are reproducible run to run); the Gram matrix B^T B is exact integer arithmetic; the k x k solve is
@@ -28,7 +37,7 @@ template <int K>
 struct QuantOut {                       // what the leader warp publishes after a reduction
     float alpha[K];
     float thr[(1 << K) - 1];
-    unsigned long long table;
+    uint32_t plane[K];                  // bit p of plane[i]: sign (1 = +1) of plane i at sorted level p
 };
 
 // Shared-memory scratch of one group (a warp, or a CTA of up to 16 warps).
@@ -217,46 +226,99 @@ __device__ __forceinline__ void level_table(const float (&alpha)[K], int lane, f
     for (int p = 0; p < M; ++p) table |= (unsigned long long)sc.code[p] << (4 * p);
 }
 
-// Quantize the vector held in w[] (elements with their bit clear in `valid` are padding and must be 0).
-// On return alpha[i] are the coefficients and bit j of bits[i] is the sign (1 = +1) of element j of this
-// thread in plane i.
+// Per-plane bit tables of the sorted code table: bit p of plane[i] = sign (1 = +1) of plane i at level p.
+template <int K>
+__device__ __forceinline__ void planes_from_table(unsigned long long table, uint32_t (&plane)[K])
+{
+#pragma unroll
+    for (int i = 0; i < K; ++i) plane[i] = 0u;
+#pragma unroll
+    for (int p = 0; p < (1 << K); ++p) {
+        const uint32_t code = (uint32_t)(table >> (4 * p)) & 15u;
+#pragma unroll
+        for (int i = 0; i < K; ++i) plane[i] |= ((code >> (K - 1 - i)) & 1u) << p;
+    }
+}
+
+// Algorithm 1 for one element: index of the leaf (sorted level) the descent over the midpoints reaches.
+// The midpoints are non-decreasing; ">=" goes to the upper half.
+template <int K>
+__device__ __forceinline__ int bst_leaf(float x, const float (&thr)[(1 << K) - 1])
+{
+    if (K == 1) return (x >= thr[0]) ? 1 : 0;
+    if (K == 2) {
+        const bool c1 = x >= thr[1];
+        const bool c2 = x >= (c1 ? thr[2] : thr[0]);
+        return (c1 ? 2 : 0) + (c2 ? 1 : 0);
+    }
+    if (K == 3) {
+        const bool c1 = x >= thr[3];
+        const bool c2 = x >= (c1 ? thr[5] : thr[1]);
+        const float hi = c2 ? thr[6] : thr[4], lo = c2 ? thr[2] : thr[0];
+        const bool c3 = x >= (c1 ? hi : lo);
+        return (c1 ? 4 : 0) + (c2 ? 2 : 0) + (c3 ? 1 : 0);
+    }
+    const bool c1 = x >= thr[7];
+    const bool c2 = x >= (c1 ? thr[11] : thr[3]);
+    const float hi3 = c2 ? thr[13] : thr[9], lo3 = c2 ? thr[5] : thr[1];
+    const bool c3 = x >= (c1 ? hi3 : lo3);
+    const float q3 = c3 ? thr[14] : thr[12], q2 = c3 ? thr[10] : thr[8];
+    const float q1 = c3 ? thr[6] : thr[4], q0 = c3 ? thr[2] : thr[0];
+    const float hi4 = c2 ? q3 : q2, lo4 = c2 ? q1 : q0;
+    const bool c4 = x >= (c1 ? hi4 : lo4);
+    return (c1 ? 8 : 0) + (c2 ? 4 : 0) + (c3 ? 2 : 0) + (c4 ? 1 : 0);
+}
+
+// Quantize the vector held in w[] (positions past the end of the vector must hold 0 and have their bit
+// clear in `valid`; `padding` is their number over the whole group).  On return alpha[i] are the
+// coefficients and bit j of bits[i] is the sign (1 = +1) of element j of this thread in plane i.
 //
 // The greedy step needs k dependent reductions (each coefficient is the mean |residue| left by the
 // previous one, Eq. 3-4); the sign plane of the last greedy bit does not depend on its own coefficient,
 // so that last reduction travels together with the sums of the first refit (Eq. 5): k + T - 1 group
 // reductions in all for T >= 1, with the values Algorithm 2 prescribes.
 template <int K, int EPT, bool MULTI>
-__device__ __forceinline__ void quantize_group(const float (&w)[EPT], uint32_t valid, int n, int T,
+__device__ __forceinline__ void quantize_group(const float (&w_in)[EPT], uint32_t valid, int n, int T,
                                                float (&alpha)[K], uint32_t (&bits)[K], QuantScratch<K>& sc)
 {
     constexpr int M = 1 << K;
     constexpr int NG = K * (K - 1) / 2;
+    constexpr uint32_t SIGN = 0x80000000u;
     const int lane = threadIdx.x & 31;
     const int nvalid = __popc(valid);
     const float inv_n = 1.0f / (float)n;
+    const float padding = (float)((MULTI ? (int)blockDim.x : 32) * EPT - n);     // zero elements past the end
     int parity = 0;
 
-    // ---- greedy initialisation, Eq. 3-4 ----
-    float last_abs = 0.0f;
+    float w[EPT];
+#pragma unroll
+    for (int j = 0; j < EPT; ++j) w[j] = w_in[j] + 0.0f;          // -0.0 -> +0.0: from here on "x >= 0" is "sign bit clear"
+
+    // ---- greedy initialisation, Eq. 3-4 (and, for T > 0, B^T w of the first refit in the same pass) ----
+    float last_abs = 0.0f, csum[K];
+    float rho = 0.0f;                                             // residue of a zero element (the padding)
     {
         float r[EPT];
 #pragma unroll
         for (int j = 0; j < EPT; ++j) r[j] = w[j];
 #pragma unroll
         for (int i = 0; i < K; ++i) {
-            float part = 0.0f;
-            uint32_t b = 0;
+            float part = 0.0f, cs = 0.0f;
+            uint32_t neg = 0;
 #pragma unroll
-            for (int j = 0; j < EPT; ++j) {
+            for (int j = EPT - 1; j >= 0; --j) {
+                const uint32_t rb = __float_as_uint(r[j]);
                 part += fabsf(r[j]);
-                if (r[j] >= 0.0f) b |= 1u << j;
+                neg = __funnelshift_l(rb, neg, 1);                // sign bit of r[j] enters at bit 0
+                cs += __uint_as_float(__float_as_uint(w[j]) ^ (rb & SIGN));        // b_i * w
             }
-            bits[i] = b & valid;
+            bits[i] = ~neg & valid;
+            csum[i] = cs;
             if (i == K - 1 && T > 0) { last_abs = part; alpha[i] = 0.0f; break; }
             float tot[1] = {part};
             int none[1] = {0};
             const bool leader = group_totals<1, 0, K, MULTI>(tot, none, sc, parity);
-            float a = tot[0] * inv_n;
+            float a = (tot[0] - padding * fabsf(rho)) * inv_n;
             if (MULTI) {
                 if (leader && lane == 0) sc.out[parity].alpha[0] = a;
                 __syncthreads();
@@ -264,26 +326,22 @@ __device__ __forceinline__ void quantize_group(const float (&w)[EPT], uint32_t v
             }
             parity ^= 1;
             alpha[i] = a;
+            const uint32_t ab = __float_as_uint(a);               // a >= 0
+            rho -= __uint_as_float(ab | (__float_as_uint(rho) & SIGN));
 #pragma unroll
             for (int j = 0; j < EPT; ++j)
-                r[j] = ((valid >> j) & 1u) ? (((b >> j) & 1u) ? r[j] - a : r[j] + a) : 0.0f;
+                r[j] -= __uint_as_float(ab | (__float_as_uint(r[j]) & SIGN));      // r - copysign(a, r)
         }
     }
 
     // ---- T alternating cycles ----
     for (int it = 0; it < T; ++it) {
-        // least-squares refit, Eq. 5: G = B^T B (exact integers), c = B^T w
+        // least-squares refit, Eq. 5: G = B^T B (exact integers), c = B^T w (summed while the codes were assigned)
         float fsum[1 + K];
         int gram[NG > 0 ? NG : 1];
         fsum[0] = last_abs;
 #pragma unroll
-        for (int i = 0; i < K; ++i) {
-            float part = 0.0f;
-#pragma unroll
-            for (int j = 0; j < EPT; ++j)
-                part += __uint_as_float(__float_as_uint(w[j]) ^ ((~(bits[i] >> j) & 1u) << 31));   // +-w
-            fsum[1 + i] = part;
-        }
+        for (int i = 0; i < K; ++i) fsum[1 + i] = csum[i];
         {
             int q = 0;
 #pragma unroll
@@ -295,50 +353,52 @@ __device__ __forceinline__ void quantize_group(const float (&w)[EPT], uint32_t v
         }
         const bool leader = group_totals<1 + K, NG, K, MULTI>(fsum, gram, sc, parity);
         float thr[M - 1];
-        unsigned long long table = 0ull;
+        uint32_t plane[K];
         if (leader) {
-            if (it == 0) alpha[K - 1] = fsum[0] * inv_n;          // the last greedy coefficient
+            if (it == 0) alpha[K - 1] = (fsum[0] - padding * fabsf(rho)) * inv_n;   // the last greedy coefficient
             float c[K];
 #pragma unroll
             for (int i = 0; i < K; ++i) c[i] = fsum[1 + i];
             solve_refit<K>(c, gram, n, alpha);
+            unsigned long long table = 0ull;
             level_table<K>(alpha, lane, thr, table, sc);
+            planes_from_table<K>(table, plane);
             if (MULTI && lane == 0) {
                 QuantOut<K>& o = sc.out[parity];
 #pragma unroll
-                for (int i = 0; i < K; ++i) o.alpha[i] = alpha[i];
+                for (int i = 0; i < K; ++i) { o.alpha[i] = alpha[i]; o.plane[i] = plane[i]; }
 #pragma unroll
                 for (int p = 0; p < M - 1; ++p) o.thr[p] = thr[p];
-                o.table = table;
             }
         }
         if (MULTI) {
             __syncthreads();
             const QuantOut<K>& o = sc.out[parity];
 #pragma unroll
-            for (int i = 0; i < K; ++i) alpha[i] = o.alpha[i];
+            for (int i = 0; i < K; ++i) { alpha[i] = o.alpha[i]; plane[i] = o.plane[i]; }
 #pragma unroll
             for (int p = 0; p < M - 1; ++p) thr[p] = o.thr[p];
-            table = o.table;
         }
         parity ^= 1;
         last_abs = 0.0f;
 
-        // Algorithm 1 for every element: leaf = number of midpoints <= w
-        const uint32_t table_lo = (uint32_t)table;
+        // Algorithm 1 for every element; the sums B^T w of the next refit are taken in the same pass
+        const bool more = it + 1 < T;
+        uint32_t pos_bits[K];
 #pragma unroll
-        for (int i = 0; i < K; ++i) bits[i] = 0;
+        for (int i = 0; i < K; ++i) { pos_bits[i] = 0u; csum[i] = 0.0f; }
 #pragma unroll
-        for (int j = 0; j < EPT; ++j) {
-            int pos = 0;
+        for (int j = EPT - 1; j >= 0; --j) {
+            const int sh = 31 - bst_leaf<K>(w[j], thr);
 #pragma unroll
-            for (int p = 0; p < M - 1; ++p) pos += (w[j] >= thr[p]) ? 1 : 0;
-            const uint32_t code = (K <= 3) ? (table_lo >> (4 * pos)) : (uint32_t)(table >> (4 * pos));
-#pragma unroll
-            for (int i = 0; i < K; ++i) bits[i] |= ((code >> (K - 1 - i)) & 1u) << j;
+            for (int i = 0; i < K; ++i) {
+                const uint32_t y = plane[i] << sh;                 // sign of plane i at this leaf, in the top bit
+                pos_bits[i] = __funnelshift_l(y, pos_bits[i], 1);
+                if (more) csum[i] += __uint_as_float(__float_as_uint(w[j]) ^ (~y & SIGN));
+            }
         }
 #pragma unroll
-        for (int i = 0; i < K; ++i) bits[i] &= valid;
+        for (int i = 0; i < K; ++i) bits[i] = pos_bits[i] & valid;
     }
 }
 
