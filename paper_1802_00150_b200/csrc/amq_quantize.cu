@@ -17,6 +17,52 @@ __device__ __forceinline__ float load_elem(const RowSource& s, int row, int t)
     return (t < s.n0) ? __ldg(s.src0 + (size_t)row * s.ld0 + t) : __ldg(s.src1 + (size_t)row * s.ld1 + (t - s.n0));
 }
 
+// Bulk variant, one row of up to 1024 elements per warp: lane l holds the 32 CONSECUTIVE elements 32 l ..
+// 32 l + 31 (eight 128-bit loads), so the sign word the quantizer leaves in a lane IS packed word l of the
+// plane and goes straight to memory, 128 contiguous bytes per warp and plane, with no ballot transposition.
+// Requires a single 16-byte-aligned source with a row stride that is a multiple of 4 elements.
+template <int K>
+__global__ void __launch_bounds__(128)
+quantize_rows_consecutive_kernel(const float* __restrict__ x, int ldx, int rows, int n, int T,
+                                 uint32_t* __restrict__ codes, float* __restrict__ coeffs)
+{
+    __shared__ QuantScratch<K> scratch[4];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int row = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (row >= rows) return;
+    const float* src = x + (size_t)row * ldx + lane * 32;
+    float w[32];
+    uint32_t valid = 0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int t = lane * 32 + q * 4;
+        float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (t + 3 < n) {
+            v = __ldcs(reinterpret_cast<const float4*>(src) + q);
+            valid |= 0xFu << (q * 4);
+        } else {
+            if (t < n) { v.x = __ldcs(src + q * 4); valid |= 1u << (q * 4); }
+            if (t + 1 < n) { v.y = __ldcs(src + q * 4 + 1); valid |= 2u << (q * 4); }
+            if (t + 2 < n) { v.z = __ldcs(src + q * 4 + 2); valid |= 4u << (q * 4); }
+        }
+        w[q * 4] = v.x; w[q * 4 + 1] = v.y; w[q * 4 + 2] = v.z; w[q * 4 + 3] = v.w;
+    }
+    float alpha[K];
+    uint32_t bits[K];
+    quantize_group<K, 32, false>(w, valid, n, T, alpha, bits, scratch[warp]);
+    const int wpr = 4 * ((n + 127) / 128);
+    if (lane < wpr) {
+#pragma unroll
+        for (int i = 0; i < K; ++i) codes[((size_t)row * K + i) * wpr + lane] = bits[i];
+    }
+    if (lane < K) {
+        float a = alpha[0];
+#pragma unroll
+        for (int i = 1; i < K; ++i) a = (lane == i) ? alpha[i] : a;
+        coeffs[(size_t)row * K + lane] = a;
+    }
+}
+
 // K bits, EPT elements per thread.  MULTI: one row per CTA (blockDim.x threads); else one row per warp.
 template <int K, int EPT, bool MULTI>
 __global__ void __launch_bounds__(256)
@@ -70,6 +116,12 @@ amq_status dispatch(const RowSource& src, int rows, int n, int T, uint32_t* code
 {
     const int n128 = 128 * ((n + 127) / 128);
     const bool bulk = rows >= 1024;
+    if (bulk && n128 > 256 && n128 <= 1024 && src.n0 == n && (src.ld0 & 3) == 0 &&
+        (reinterpret_cast<uintptr_t>(src.src0) & 15u) == 0) {
+        quantize_rows_consecutive_kernel<K><<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(src.src0, src.ld0, rows, n, T, codes, coeffs);
+        AMQ_LAUNCH_CHECK();
+        return AMQ_OK;
+    }
     if (bulk && n128 <= 256) return run<K, 8, false>(src, rows, n, T, codes, coeffs, 128, st);
     if (bulk && n128 <= 1024) return run<K, 32, false>(src, rows, n, T, codes, coeffs, 128, st);
     if (bulk || n128 > 2048) {
