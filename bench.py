@@ -82,7 +82,7 @@ def oracle_setup(wl, rows_limit=None):
     return Wc, Wa
 
 
-def oracle_step(wl, Wc, Wa, ins, batch_limit=None):
+def oracle_step(wl, Wc, Wa, ins, batch_limit=None, timestep_limit=None):
     """One benchmark step on the oracle; returns the number of units (timesteps x sequences) it covered."""
     import oracle
     if wl.cell == "proj":
@@ -91,12 +91,13 @@ def oracle_step(wl, Wc, Wa, ins, batch_limit=None):
         oracle.binary_gemm(Wc, Wa, Xc, Xb, wl.n)
         return acts.shape[0] / wl.batch * (Wc.shape[0] / wl.m)
     b = wl.batch if batch_limit is None else min(batch_limit, wl.batch)
-    xs, h0, c0 = ins["x_seq"][:, :b], ins["h0"][:b], ins["c0"][:b]
+    ts = wl.steps if timestep_limit is None else max(1, min(timestep_limit, wl.steps))
+    xs, h0, c0 = ins["x_seq"][:ts, :b], ins["h0"][:b], ins["c0"][:b]
     if wl.cell == "lstm":
         oracle.lstm_sequence(Wc, Wa, None, wl.I, wl.H, xs, h0, c0, wl.k_a, wl.T)
     else:
         oracle.gru_sequence(Wc, Wa, None, wl.I, wl.H, xs, h0, wl.k_a, wl.T)
-    return wl.steps * b
+    return ts * b
 
 
 def oracle_sample_plan(wl):
@@ -115,12 +116,22 @@ def run_reference(args, wl):
     rows_limit, batch_limit, desc = oracle_sample_plan(wl)
     Wc, Wa = oracle_setup(wl, rows_limit)
     ins = synth.inputs(wl)
+    # keep the whole run within a few minutes: if K full samples would not fit, each step covers only the
+    # first timesteps of the sequence (the sample is described in the output)
+    t0 = time.perf_counter()
+    oracle_step(wl, Wc, Wa, ins, batch_limit)
+    t_one = time.perf_counter() - t0
+    ts_limit = None
+    budget_s = 150.0
+    if wl.cell != "proj" and (args.steps + args.warmup) * t_one > budget_s:
+        ts_limit = max(1, int(wl.steps * budget_s / ((args.steps + args.warmup) * t_one)))
+        desc += "; first %d of %d timesteps per step (time budget)" % (min(ts_limit, wl.steps), wl.steps)
     for _ in range(args.warmup):
-        oracle_step(wl, Wc, Wa, ins, batch_limit)
+        oracle_step(wl, Wc, Wa, ins, batch_limit, ts_limit)
     units = 0.0
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        units += oracle_step(wl, Wc, Wa, ins, batch_limit)
+        units += oracle_step(wl, Wc, Wa, ins, batch_limit, ts_limit)
     dt = time.perf_counter() - t0
     value = units / dt if wl.cell != "proj" else units / dt
     unit = "timesteps/s" if wl.cell != "proj" else "passes/s"
