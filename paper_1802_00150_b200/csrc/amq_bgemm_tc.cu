@@ -5,9 +5,8 @@
 // with the row-wise coefficients afterwards (Sec. 4), and for the cells the gate arithmetic of Eq. 6 /
 // the GRU follows in the same kernel.
 //
-// The planes stay bit-packed in global memory.  A CTA expands the bits of its tile into signed bytes on chip
-// (the weight operand into tensor memory, the activation operand into shared memory, so that the two do not
-// compete for the shared-memory port): bit 1 -> -64, bit 0 -> +64 on both operands, so a byte product is 4096 * (+-1 * +-1) and a
+// The planes stay bit-packed in global memory.  A CTA expands the bits of its tile into signed bytes in
+// shared memory: bit 1 -> -64, bit 0 -> +64 on both operands, so a byte product is 4096 * (+-1 * +-1) and a
 // 32-bit accumulator holds 4096 * (dot of the +-1 vectors); pad positions (0 in both operands) add one
 // each and are subtracted again.  Expanding costs one shift (issued as a multiplication, on the FMA pipe)
 // and one three-input logic operation per four bytes: output register s of a 32-bit word keeps bits s,
@@ -15,9 +14,7 @@
 // both operands, which a dot product does not see.  What bounds the expansion is the shared-memory store
 // bandwidth (128 operand bytes per row and stage), not the arithmetic.
 //
-// Weight operand (A) in tensor memory: lane = row of the M tile, a pipeline stage = 32 consecutive 32-bit
-// columns = 128 bytes of K, written by the row's thread with tcgen05.st; an MMA takes 8 columns.
-// Activation operand (B) in shared memory, K-major with the 128-byte swizzle: a pipeline stage holds 128 bytes of K per
+// Shared-memory operand layout: K-major with the 128-byte swizzle: a pipeline stage holds 128 bytes of K per
 // operand row, rows are 128 bytes apart, groups of 8 rows 1024 bytes apart, and the 16-byte chunk j of row r
 // sits at chunk position j xor (r mod 8).  One MMA instruction consumes K = 32 bytes = the two chunks of one
 // packed word; its descriptor start address advances by 32 bytes per word inside the swizzled row.
@@ -55,9 +52,7 @@ struct TcParams {
     int nseg;       // 1, or 2 for the GRU (columns [0,I) and [I,n))
     int wpr;
     int n_mma;      // TB * k_a: N of the MMA, multiple of 16, <= 256
-    int tmem_cols;  // power of two >= accumulators (MT * nseg * n_mma columns) + weight-operand stages
-    int bar_off;    // byte offset of the mbarriers in dynamic shared memory (past the operand stages / epilogue tiles)
-    int a_col0;     // first tensor-memory column of the weight-operand stages (32 columns per M tile and stage)
+    int tmem_cols;  // power of two >= MT * nseg * n_mma
     int nstages;    // pipeline depth
     int expanders;  // operand rows of a stage, MT * 128 + n_mma, rounded up to whole warps
     int groups;     // expander groups (1 or 2) that take the pipeline steps in turn, `expanders` threads each
@@ -112,21 +107,13 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
     return (uint64_t)((addr >> 4) & 0x3fffu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
-// D (tensor memory) (+)= A (tensor memory: 128 lanes = rows, K = 32 bytes in 8 consecutive 32-bit columns) x B (shared memory)
-__device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
-        :: "r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-// eight consecutive 32-bit columns of this thread's lane of tensor memory
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&v)[8])
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 :: "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
 __device__ __forceinline__ void mma_commit(uint32_t bar)
@@ -178,12 +165,12 @@ bgemm_tc_kernel(TcParams p)
     const int EXP = p.expanders;                    // operand rows rounded up to whole warps
     const int mma_warp = (G * EXP) >> 5, nthreads = G * EXP + 32;
     const int n_mma = p.n_mma;
-    const int stage_bytes = n_mma * 128;            // activation operand: 128 bytes of K per row and stage, in shared memory
-    const int a_stage_cols = MT * 32;               // weight operand: 128 bytes of K per row and stage = 32 columns of tensor memory per M tile
+    const int a_stage_bytes = MT * TILE_M * 128;    // 128 bytes of K per row and stage
+    const int stage_bytes = a_stage_bytes + n_mma * 128;
     const int u0 = blockIdx.x * p.UT * MT, b0 = blockIdx.y * p.TB;
 
     unsigned char* stage_base = smem_raw;
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw + p.bar_off);                 // [S]
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)S * stage_bytes);   // [S]
     uint64_t* empty_bar = full_bar + MAX_STAGES;                                            // [S]
     uint64_t* done_bar = empty_bar + MAX_STAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done_bar + 1);
@@ -225,18 +212,14 @@ bgemm_tc_kernel(TcParams p)
                 if (u < p.units)
                     src = reinterpret_cast<const uint4*>(a.Wcodes + (((size_t)gate * p.units + u) * k_w + i) * p.wpr);
             }
-            dst0 = 0;
+            dst0 = smem_u32(stage_base) + r_all * 128;
         } else {
             const int r = r_all - MT * TILE_M;
             const int b = b0 + r / KA, j = r % KA;
             if (r < n_mma && b < a.batch) src = reinterpret_cast<const uint4*>(a.xcodes + ((size_t)b * KA + j) * p.wpr);
-            dst0 = smem_u32(stage_base) + r * 128;
+            dst0 = smem_u32(stage_base) + a_stage_bytes + r * 128;
         }
         const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
-        // weight rows go to tensor memory: whole warps (EXP is a multiple of 128, so warp w of a group owns lane
-        // quarter w mod 4 of M tile w / 4); activation rows go to shared memory
-        const bool to_tmem = r_all < MT * TILE_M;
-        const uint32_t a_t0 = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(p.a_col0 + (r_all >> 7) * 32);
         uint32_t off[8];                                            // swizzled position of chunk j: j xor (row mod 8)
 #pragma unroll
         for (int j = 0; j < 8; ++j) off[j] = (uint32_t)((j ^ (r_all & 7)) << 4);
@@ -254,23 +237,9 @@ bgemm_tc_kernel(TcParams p)
             const uint4 v = cur;
             cur = nxt;
             nxt = (src && c + 2 * G < CH) ? __ldg(src + c + 2 * G) : zero;
-            // the MMAs that read this buffer one lap ago must have completed (the outcome is made uniform over
-            // the warp: the tensor-memory stores below are warp-wide instructions)
-            if (!__all_sync(0xffffffffu, mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity))) { *failed = 1; break; }
-            if (to_tmem) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint32_t y[8];
-#pragma unroll
-                    for (int s = 0; s < 7; ++s) y[s] = and_xor(w[q] * mul[s], m_sign, m_half);     // w << (7 - s)
-                    y[7] = and_xor(w[q], m_sign, m_half);
-                    tmem_st8(a_t0 + (uint32_t)(buf * a_stage_cols + q * 8), y);
-                }
-                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            } else if (writes) {
+            // the MMAs that read this buffer one lap ago must have completed
+            if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; break; }
+            if (writes) {
                 const uint32_t base = dst0 + (uint32_t)(buf * stage_bytes);
                 const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -283,7 +252,7 @@ bgemm_tc_kernel(TcParams p)
                     st_shared_v4(base + off[2 * q + 1], y[4], y[5], y[6], y[7]);
                 }
             }
-            if (!to_tmem) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
             buf += G;
             if (buf >= S) { buf -= S; empty_parity ^= 1u; }
@@ -298,16 +267,16 @@ bgemm_tc_kernel(TcParams p)
             if (!mbar_wait(smem_u32(&full_bar[buf]), full_parity)) { *failed = 1; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             // descriptors of the stage: start addresses are below 256 KiB, so adding to the low word never carries
-            const uint64_t bdesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
-            const uint32_t a_t = tmem_base + (uint32_t)(p.a_col0 + buf * a_stage_cols);
+            const uint64_t adesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
+            const uint64_t bdesc0 = adesc0 + (uint64_t)(a_stage_bytes >> 4);
 #pragma unroll
             for (int qq = 0; qq < STAGE_WORDS; ++qq) {
                 const int word = c * STAGE_WORDS + qq;
                 const int seg = word >= split_word ? 1 : 0;
                 const uint32_t accumulate = (word != 0 && word != split_word) ? 1u : 0u;
-                mma_i8_ts(tmem_base + seg * n_mma, a_t + qq * 8, bdesc0 + 2 * qq, idesc, accumulate);
+                mma_i8(tmem_base + seg * n_mma, adesc0 + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
                 if (MT == 2)
-                    mma_i8_ts(tmem_base + (p.nseg + seg) * n_mma, a_t + 32 + qq * 8, bdesc0 + 2 * qq, idesc, accumulate);
+                    mma_i8(tmem_base + (p.nseg + seg) * n_mma, adesc0 + (TILE_M * 128 >> 4) + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
             }
             mma_commit(smem_u32(&empty_bar[buf]));
             if (++buf == S) { buf = 0; full_parity ^= 1u; }
@@ -490,38 +459,34 @@ bool plan(const GemmArgs& a, TcPlan* out)
     } else { p.gates = 1; p.units = a.m; }
     p.UT = TILE_M / (p.gates * a.k_w);
     if (p.UT < 1) return false;
-    // batch entries per tile: multiples of 16, N = TB * k_a <= 256; tensor memory (512 columns) holds the
-    // accumulators (nseg * N per M tile) and MAX_STAGES stages of the weight operand (32 columns per M tile)
-    const int S = MAX_STAGES;
-    int n_max = (512 - S * 32) / p.nseg;
-    if (n_max > 256) n_max = 256;
-    int tb_max = (n_max / a.k_a) / 16 * 16;
+    // batch entries per tile: multiples of 16, N = TB * k_a <= 256
+    int tb_max = (256 / a.k_a) / 16 * 16;
     if (tb_max > 128) tb_max = 128;
-    if (tb_max < 16) return false;
     const int ntiles = (a.batch + tb_max - 1) / tb_max;
     p.TB = ((a.batch + ntiles - 1) / ntiles + 15) / 16 * 16;
     p.n_mma = p.TB * a.k_a;
-    // two M tiles per CTA when tensor memory allows and enough CTAs remain to fill the GPU
+    // two M tiles per CTA when their accumulators fit tensor memory and enough CTAs remain to fill the GPU
     const int mtiles = (p.units + p.UT - 1) / p.UT;
     const int btiles = (a.batch + p.TB - 1) / p.TB;
-    p.MT = (2 * (p.nseg * p.n_mma + S * 32) <= 512 && (long long)(mtiles / 2) * btiles >= 2 * 148) ? 2 : 1;
-    p.a_col0 = p.MT * p.nseg * p.n_mma;
+    p.MT = (2 * p.nseg * p.n_mma <= 512 && (long long)(mtiles / 2) * btiles >= 2 * 148) ? 2 : 1;
     int cols = 32;
-    while (cols < p.a_col0 + S * p.MT * 32) cols <<= 1;
+    while (cols < p.MT * p.nseg * p.n_mma) cols <<= 1;
     if (cols > 512) return false;
     p.tmem_cols = cols;
-    p.expanders = (p.MT * TILE_M + p.n_mma + 127) / 128 * 128;
-    const size_t stage = (size_t)128 * p.n_mma;
+    const size_t stage = (size_t)128 * (p.MT * TILE_M + p.n_mma);
     const size_t epi = ((size_t)p.MT * p.nseg * TILE_M * (p.TB + 1) + (size_t)p.TB * a.k_a) * 4;
-    const size_t buffers = S * stage > epi ? S * stage : epi;
+    int S = (int)((220 * 1024) / stage);
+    if (S > MAX_STAGES) S = MAX_STAGES;
+    if (S < 2) return false;
+    if (epi > S * stage) return false;
     p.nstages = S;
+    p.expanders = (p.MT * TILE_M + p.n_mma + 31) / 32 * 32;
     p.groups = (2 * p.expanders + 32 <= MAX_THREADS) ? 2 : 1;
     for (int sft = 0; sft < 8; ++sft) p.mul[sft] = 1u << (7 - sft);
     p.mask_sign = 0x80808080u;
     p.mask_half = 0x40404040u;
-    p.bar_off = (int)((buffers + 1023) / 1024 * 1024);
     out->p = p;
-    out->smem = (size_t)p.bar_off + (2 * MAX_STAGES + 1) * 8 + 16;
+    out->smem = S * stage + (2 * MAX_STAGES + 1) * 8 + 16;
     out->grid = dim3((unsigned)((mtiles + p.MT - 1) / p.MT), (unsigned)btiles);
     return out->grid.y <= 65535u && out->smem <= 227 * 1024;
 }
