@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by workload; the summaries are under profiles/.  None = not captured.
-NCU_TRAFFIC_BYTES = {"lstm1024_b1": 2331904 + 8192}     # rnn_persistent_kernel, profiles/rnn_persistent_kernel_lstm1024_b1.txt
+NCU_TRAFFIC_BYTES = {"lstm1024_b1": 2331648 + 10496}     # rnn_persistent_kernel, profiles/rnn_persistent_kernel_lstm1024_b1.txt
 
 
 def parse_args():
