@@ -505,8 +505,11 @@ amq_status launch_ka(const TcPlan& pl, cudaStream_t st)
 
 bool gemm_tc_supported(const GemmArgs& a)
 {
+    // from 16 vectors on always; for 2..15 vectors (one padded tile of 16) when the weight matrix is large
+    // enough that the CUDA-core kernel's tile loop costs more than this kernel's fixed ~10 us
     TcPlan pl;
-    return a.batch >= 16 && plan(a, &pl);
+    const bool big = (long long)a.m * a.k_w * words_per_row(a.n) >= (1ll << 17);
+    return (a.batch >= 16 || (a.batch >= 2 && big)) && plan(a, &pl);
 }
 
 amq_status launch_binary_gemm_tc(const GemmArgs& a, cudaStream_t st)

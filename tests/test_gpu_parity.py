@@ -149,6 +149,8 @@ GEMM_CASES = [
     (33, 31, 1, 1, 3),
     (257, 300, 1, 4, 17),
     (40, 8192, 2, 2, 2),
+    (2048, 2048, 2, 2, 5),               # few vectors, large matrix: one padded tile on the tensor cores
+    (1031, 4096, 3, 2, 15),
     # batch 1: the streaming matrix-vector kernel (segments of 1..32 lanes per row, one or two chunks per lane)
     (300, 8192, 3, 3, 1),
     (1000, 1024, 2, 3, 1),
