@@ -49,6 +49,8 @@ _gemm = _sig("amq_oracle_binary_gemm_range", None, _u32p, _dp, _int, _int, _int,
              _dp, _int, _int, _dp)
 _lstm = _sig("amq_oracle_lstm_step", None, _u32p, _dp, _dp, _int, _int, _int, _dp, _dp, _dp, _int, _int, _int,
              _dp, _dp)
+_lstm_paper = _sig("amq_oracle_lstm_step_paper", None, _u32p, _dp, _u32p, _dp, _dp, _int, _int, _int, _u32p, _dp, _int,
+                   _dp, _dp, _int, _int, _int, _dp, _dp)
 _gru = _sig("amq_oracle_gru_step", None, _u32p, _dp, _dp, _int, _int, _int, _dp, _dp, _int, _int, _int, _dp)
 _lstm_seq = _sig("amq_oracle_lstm_sequence", None, _u32p, _dp, _dp, _int, _int, _int, _dp, _int, _dp, _dp,
                  _int, _int, _int, _dp, _dp, _dp)
@@ -213,6 +215,20 @@ def lstm_step(Wcodes, Walpha, bias, I, H, x, h, c, k_a, T):
     h_out, c_out = np.zeros((batch, H)), np.zeros((batch, H))
     _lstm(_p(Wc, _u32p), _p(Wa, _dp), _p(bias, _dp), I, H, k_w, _p(x, _dp), _p(h, _dp), _p(c, _dp),
           batch, k_a, T, _p(h_out, _dp), _p(c_out, _dp))
+    return h_out, c_out
+
+
+def lstm_step_paper(Wi_codes, Wi_alpha, Wh_codes, Wh_alpha, bias, I, H, xcodes, xbeta, h, c, k_a, T):
+    """The step as the paper states it: separate W_i / W_h, x given as packed codes (an embedding row), h quantized on-line."""
+    Wic = np.ascontiguousarray(Wi_codes, dtype=np.uint32)
+    Whc = np.ascontiguousarray(Wh_codes, dtype=np.uint32)
+    xc = np.ascontiguousarray(xcodes, dtype=np.uint32)
+    Wia, Wha, xb, h, c = _d(Wi_alpha), _d(Wh_alpha), _d(xbeta), _d(h), _d(c)
+    k_w, (batch, k_e, _) = Wic.shape[1], xc.shape
+    bias = None if bias is None else _d(bias)
+    h_out, c_out = np.zeros((batch, H)), np.zeros((batch, H))
+    _lstm_paper(_p(Wic, _u32p), _p(Wia, _dp), _p(Whc, _u32p), _p(Wha, _dp), _p(bias, _dp), I, H, k_w,
+                _p(xc, _u32p), _p(xb, _dp), k_e, _p(h, _dp), _p(c, _dp), batch, k_a, T, _p(h_out, _dp), _p(c_out, _dp))
     return h_out, c_out
 
 

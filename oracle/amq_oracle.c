@@ -360,6 +360,43 @@ void amq_oracle_lstm_step(const uint32_t* Wcodes, const double* Walpha, const do
 }
 
 /* ---------------------------------------------------------------------------------------------
+ * One quantized LSTM step in the form the paper states it (Eq. 6 and the text after it): two weight
+ * matrices W_i (4H x I) and W_h (4H x H), each quantized row by row on its own; x_t is a row of the
+ * quantized embedding W_e and "needs no more quantization", so it arrives as k_e packed planes with
+ * coefficients; only h_{t-1} is quantized on-line (k_a bits, T cycles).
+ *   p = W_i_hat x_hat + W_h_hat h_hat + bias;  i, f, o = logistic(p), g = tanh(p) (gate order i, f, o, g);
+ *   c' = f * c + i * g;  h' = o * tanh(c').
+ * xcodes [batch][k_e][wpr(I)], xbeta [batch][k_e]; h/c [batch][H] double; bias 4H or NULL.
+ * ------------------------------------------------------------------------------------------- */
+void amq_oracle_lstm_step_paper(const uint32_t* Wi_codes, const double* Wi_alpha,
+                                const uint32_t* Wh_codes, const double* Wh_alpha, const double* bias,
+                                int I, int H, int k_w, const uint32_t* xcodes, const double* xbeta, int k_e,
+                                const double* h_in, const double* c_in, int batch, int k_a, int T,
+                                double* h_out, double* c_out)
+{
+    int m = 4 * H, wpr_i = amq_oracle_words_per_row(I), wpr_h = amq_oracle_words_per_row(H);
+    double* pi = (double*)malloc(sizeof(double) * (size_t)m);
+    double* ph = (double*)malloc(sizeof(double) * (size_t)m);
+    uint32_t* hc = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)k_a * wpr_h);
+    double beta[AMQ_ORACLE_MAX_K];
+    for (int bt = 0; bt < batch; ++bt) {
+        amq_oracle_quantize_rows(h_in + (size_t)bt * H, 1, H, H, k_a, T, hc, beta);
+        amq_oracle_binary_gemm(Wi_codes, Wi_alpha, m, I, k_w, xcodes + (size_t)bt * k_e * wpr_i,
+                               xbeta + (size_t)bt * k_e, 1, k_e, NULL, pi);
+        amq_oracle_binary_gemm(Wh_codes, Wh_alpha, m, H, k_w, hc, beta, 1, k_a, NULL, ph);
+        for (int u = 0; u < H; ++u) {
+            double p4[4];
+            for (int g = 0; g < 4; ++g) p4[g] = pi[g * H + u] + ph[g * H + u] + (bias ? bias[g * H + u] : 0.0);
+            double ig = logistic(p4[0]), fg = logistic(p4[1]), og = logistic(p4[2]), gg = tanh(p4[3]);
+            double c = fg * c_in[(size_t)bt * H + u] + ig * gg;
+            c_out[(size_t)bt * H + u] = c;
+            h_out[(size_t)bt * H + u] = og * tanh(c);
+        }
+    }
+    free(pi); free(ph); free(hc);
+}
+
+/* ---------------------------------------------------------------------------------------------
  * One quantized GRU step.  The paper names the GRU but prints no equations; this is the common
  * "linear before reset" form (a stated reading, not the paper's text):
  *   W: 3H rows in the order r, z, n; p = W_hat z_hat with z_hat the quantized [x ; h];

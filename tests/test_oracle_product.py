@@ -221,3 +221,38 @@ def test_synth_is_reproducible_and_shaped():
     assert (wl.m, wl.n) == (4096, 2048)
     ins = synth.inputs(wl)
     assert ins["x_seq"].shape == (35, 1, 1024) and np.abs(ins["x_seq"]).max() <= 3.0
+
+
+@pytest.mark.parametrize("I,H,batch,kw,ke,ka", [(20, 12, 2, 2, 2, 2), (33, 31, 1, 3, 2, 3), (64, 40, 3, 2, 3, 1)])
+def test_paper_form_lstm_step_equals_textbook_step_on_reconstructed_operands(I, H, batch, kw, ke, ka):
+    """Eq. 6 as printed: separate W_i and W_h, x an (already quantized) embedding row, only h quantized on-line."""
+    Wi = synth.normal((4 * H, I), 0.2, 17, 1).astype(np.float64)
+    Wh = synth.normal((4 * H, H), 0.2, 17, 2).astype(np.float64)
+    bias = synth.normal((4 * H,), 0.1, 17, 3).astype(np.float64)
+    emb = synth.normal((batch, I), 0.5, 17, 4).astype(np.float64)          # the embedding rows of the tokens
+    h = synth.uniform((batch, H), -1, 1, 17, 5).astype(np.float64)
+    c = synth.uniform((batch, H), -1, 1, 17, 6).astype(np.float64)
+    Wic, Wia = oracle.quantize_rows(Wi, kw, 2)
+    Whc, Wha = oracle.quantize_rows(Wh, kw, 2)
+    xc, xb = oracle.quantize_rows(emb, ke, 2)                              # offline, like every row of W_e
+    hc, hb = oracle.quantize_rows(h, ka, 2)
+    # textbook step on the dense reconstructions, with the stacked matrix [W_i | W_h]
+    What = np.concatenate([dense_hat(Wic, Wia, I), dense_hat(Whc, Wha, H)], axis=1)
+    h_ref, c_ref = textbook_lstm(What, bias, dense_hat(xc, xb, I), dense_hat(hc, hb, H), c, H)
+    h_out, c_out = oracle.lstm_step_paper(Wic, Wia, Whc, Wha, bias, I, H, xc, xb, h, c, ka, 2)
+    assert np.allclose(h_out, h_ref, rtol=1e-11, atol=1e-13) and np.allclose(c_out, c_ref, rtol=1e-11, atol=1e-13)
+
+
+def test_paper_form_lstm_step_reduces_to_full_precision_when_two_bits_are_exact():
+    I, H, batch = 24, 16, 2
+    x = exactly_representable((batch, I), 0.5, 0.125, 19, 1)
+    h = exactly_representable((batch, H), 0.25, 0.0625, 19, 2)
+    c = synth.uniform((batch, H), -1, 1, 19, 3).astype(np.float64)
+    Wi = exactly_representable((4 * H, I), 0.05, 0.02, 19, 4)
+    Wh = exactly_representable((4 * H, H), 0.07, 0.01, 19, 5)
+    Wic, Wia = oracle.quantize_rows(Wi, 2, 2)
+    Whc, Wha = oracle.quantize_rows(Wh, 2, 2)
+    xc, xb = oracle.quantize_rows(x, 2, 2)
+    h_out, c_out = oracle.lstm_step_paper(Wic, Wia, Whc, Wha, None, I, H, xc, xb, h, c, 2, 2)
+    h_ref, c_ref = textbook_lstm(np.concatenate([Wi, Wh], axis=1), None, x, h, c, H)
+    assert np.allclose(h_out, h_ref, atol=1e-12) and np.allclose(c_out, c_ref, atol=1e-12)
