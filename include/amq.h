@@ -205,6 +205,49 @@ AMQ_API amq_status amq_gru_sequence(const uint32_t* Wcodes, const float* Walpha,
                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The LSTM in the form the paper states it (Eq. 6 and the paragraph after it): separate matrices W_i (4H x I)
+ * and W_h (4H x H), each quantized row by row; x_t is a row of the quantized embedding matrix and needs no
+ * further quantization; only h_{t-1} is quantized on-line.
+ *
+ * amq_embedding_rows: x_t = W_e^T y*_{t-1} for one-hot tokens = gather of rows of the quantized W_e.
+ *   We_codes [vocab][k][wpr(n)], We_alpha [vocab][k]; tokens [count] int32 (ids outside [0, vocab) are clamped);
+ *   xcodes [count][k][wpr(n)], xbeta [count][k] out.
+ */
+AMQ_API amq_status amq_embedding_rows(const uint32_t* We_codes, const float* We_alpha, int vocab, int n, int k,
+                              const int32_t* tokens, int count, uint32_t* xcodes, float* xbeta, void* stream);
+
+/* Scratch of the two calls below, in bytes (steps = 1 for the step call); 0 on invalid arguments. */
+AMQ_API size_t amq_lstm_paper_workspace_bytes(int H, int batch, int steps, int k_a);
+
+/*
+ * One step:  p = W_i_hat x_hat + W_h_hat h_hat + bias, gates as in amq_lstm_step (order i, f, o, g).
+ *   Wi_codes [4H][k_w][wpr(I)], Wi_alpha [4H][k_w]; Wh_codes [4H][k_w][wpr(H)], Wh_alpha [4H][k_w]; bias [4H] or NULL.
+ *   xcodes [batch][k_e][wpr(I)], xbeta [batch][k_e]: the inputs, already quantized (k_e bits).
+ *   h_in is quantized on-line with k_a bits and T cycles.  h_out must not alias h_in; c_out may alias c_in.
+ */
+AMQ_API amq_status amq_lstm_step_paper(const uint32_t* Wi_codes, const float* Wi_alpha,
+                               const uint32_t* Wh_codes, const float* Wh_alpha, const float* bias,
+                               int I, int H, int k_w,
+                               const uint32_t* xcodes, const float* xbeta, int k_e,
+                               const float* h_in, const float* c_in, int batch, int k_a, int T,
+                               float* h_out, float* c_out,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * `steps` consecutive steps.  xcodes_seq [steps][batch][k_e][wpr(I)], xbeta_seq [steps][batch][k_e].
+ * The input projections W_i x_t + bias of all timesteps do not depend on the state and are computed by one
+ * batched binary product before the time loop; each timestep then quantizes h and multiplies by W_h only.
+ * h_seq [steps][batch][H] out or NULL; h_last, c_last [batch][H] out; outputs must not alias inputs.
+ */
+AMQ_API amq_status amq_lstm_sequence_paper(const uint32_t* Wi_codes, const float* Wi_alpha,
+                                   const uint32_t* Wh_codes, const float* Wh_alpha, const float* bias,
+                                   int I, int H, int k_w,
+                                   const uint32_t* xcodes_seq, const float* xbeta_seq, int k_e, int steps,
+                                   const float* h0, const float* c0, int batch, int k_a, int T,
+                                   float* h_seq, float* h_last, float* c_last,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The sequence calls with HOST activations and results: x_seq, h0, c0 are read from host memory
  * (pinned memory makes the copies asynchronous) into `staging`, the sequence runs, and h_last / c_last
  * (and h_seq when not NULL) are copied back to host memory; the call returns after the stream has

@@ -52,6 +52,12 @@ EXPORTS = {
     "amq_gru_sequence_host": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _int, _vp, _int, _int, _int,
                                      _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
     "amq_workspace_status": (_int, [_vp, _vp]),
+    "amq_embedding_rows": (_int, [_vp, _vp, _int, _int, _int, _vp, _int, _vp, _vp, _vp]),
+    "amq_lstm_paper_workspace_bytes": (_sz, [_int, _int, _int, _int]),
+    "amq_lstm_step_paper": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _int, _int, _vp, _vp, _int, _vp, _vp, _int, _int, _int,
+                                   _vp, _vp, _vp, _sz, _vp]),
+    "amq_lstm_sequence_paper": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _int, _int, _vp, _vp, _int, _int, _vp, _vp, _int, _int,
+                                       _int, _vp, _vp, _vp, _vp, _sz, _vp]),
 }
 
 for _name, (_res, _args) in EXPORTS.items():
@@ -286,3 +292,44 @@ def gru_sequence_host(Wcodes, Walpha, bias, I, H, x_seq, h0, k_a, T, workspace, 
 
 def workspace_status(workspace):
     return _lib.amq_workspace_status(_ptr(workspace), _stream())
+
+
+def embedding_rows(We_codes, We_alpha, n, tokens):
+    """Rows of the quantized embedding matrix for int32 token ids of any shape -> codes (*shape, k, wpr), coeffs (*shape, k)."""
+    We_codes, We_alpha = _dev(We_codes, torch.int32, "We_codes"), _dev(We_alpha, torch.float32, "We_alpha")
+    tokens = _dev(tokens, torch.int32, "tokens")
+    vocab, k, wpr = We_codes.shape
+    xcodes = torch.empty(tuple(tokens.shape) + (k, wpr), dtype=torch.int32, device=We_codes.device)
+    xbeta = torch.empty(tuple(tokens.shape) + (k,), dtype=torch.float32, device=We_codes.device)
+    _check(_lib.amq_embedding_rows(_ptr(We_codes), _ptr(We_alpha), vocab, n, k, _ptr(tokens), tokens.numel(),
+                                   _ptr(xcodes), _ptr(xbeta), _stream()))
+    return xcodes, xbeta
+
+
+def new_paper_workspace(H, batch, steps, k_a, device="cuda"):
+    return torch.empty(max(_lib.amq_lstm_paper_workspace_bytes(H, batch, steps, k_a), 16), dtype=torch.uint8, device=device)
+
+
+def lstm_step_paper(Wi_codes, Wi_alpha, Wh_codes, Wh_alpha, bias, I, H, xcodes, xbeta, h_in, c_in, k_a, T, workspace,
+                    h_out=None, c_out=None):
+    batch, k_w, k_e = h_in.shape[0], Wi_codes.shape[1], xcodes.shape[-2]
+    h_out = torch.empty_like(h_in) if h_out is None else h_out
+    c_out = torch.empty_like(c_in) if c_out is None else c_out
+    _check(_lib.amq_lstm_step_paper(_ptr(Wi_codes), _ptr(Wi_alpha), _ptr(Wh_codes), _ptr(Wh_alpha), _ptr(bias), I, H, k_w,
+                                    _ptr(xcodes), _ptr(xbeta), k_e, _ptr(h_in), _ptr(c_in), batch, k_a, T,
+                                    _ptr(h_out), _ptr(c_out), _ptr(workspace), workspace.numel(), _stream()))
+    return h_out, c_out
+
+
+def lstm_sequence_paper(Wi_codes, Wi_alpha, Wh_codes, Wh_alpha, bias, I, H, xcodes_seq, xbeta_seq, h0, c0, k_a, T, workspace,
+                        want_h_seq=False, h_last=None, c_last=None):
+    steps, batch, k_e = xcodes_seq.shape[0], h0.shape[0], xcodes_seq.shape[-2]
+    k_w = Wi_codes.shape[1]
+    h_seq = torch.empty((steps, batch, H), dtype=torch.float32, device=h0.device) if want_h_seq else None
+    h_last = torch.empty_like(h0) if h_last is None else h_last
+    c_last = torch.empty_like(c0) if c_last is None else c_last
+    _check(_lib.amq_lstm_sequence_paper(_ptr(Wi_codes), _ptr(Wi_alpha), _ptr(Wh_codes), _ptr(Wh_alpha), _ptr(bias), I, H, k_w,
+                                        _ptr(xcodes_seq), _ptr(xbeta_seq), k_e, steps, _ptr(h0), _ptr(c0), batch, k_a, T,
+                                        _ptr(h_seq), _ptr(h_last), _ptr(c_last), _ptr(workspace), workspace.numel(),
+                                        _stream()))
+    return h_seq, h_last, c_last

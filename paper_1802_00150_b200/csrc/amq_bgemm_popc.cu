@@ -164,7 +164,8 @@ bgemm_popc_kernel(PopcParams p)
                 float pre[4];
 #pragma unroll
                 for (int g = 0; g < 4; ++g)
-                    pre[g] = Yt[(ul * 4 + g) * p.TB + bb] + (a.bias ? __ldg(a.bias + g * H + u) : 0.0f);
+                    pre[g] = Yt[(ul * 4 + g) * p.TB + bb] + (a.bias ? __ldg(a.bias + g * H + u) : 0.0f) +
+                             (a.addend ? __ldg(a.addend + (size_t)b * a.ld_addend + g * H + u) : 0.0f);
                 const float ig = logistic(pre[0]), fg = logistic(pre[1]), og = logistic(pre[2]);
                 const float gg = tanhf(pre[3]);
                 const size_t o = (size_t)b * H + u;

@@ -404,6 +404,7 @@ bgemm_tc_kernel(TcParams p)
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     float s = bias4[g];
+                    if (a.addend) s += __ldg(a.addend + (size_t)(b0 + bb) * a.ld_addend + g * H + u);
                     for (int i = 0; i < k_w; ++i) s += y0[(g * k_w + i) * ldy + bb];
                     g4[g] = s;
                 }

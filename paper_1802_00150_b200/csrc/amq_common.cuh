@@ -84,6 +84,9 @@ struct GemmArgs {
     // EPI_LSTM / EPI_GRU
     int I, H;
     const float* h_in; const float* c_in; float* h_out; float* c_out;
+    // EPI_LSTM only: optional pre-activations computed elsewhere (e.g. W_i x), added before the gates;
+    // addend[b * ld_addend + gate * H + unit]
+    const float* addend; int ld_addend;
 };
 
 amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st);
