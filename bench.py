@@ -512,7 +512,37 @@ def batched_lines(amq, torch, dev, flush, hbm_peak, peak_kind):
                         "ms": msb, "bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": hbm_peak, "frac": gbs / hbm_peak,
                         "peak_kind": "of " + peak_kind, "algorithmic_bytes": int(alg)})
         del W, Wcodes, Walpha, acts, xc, xb, y
+    out.append(paper_form_line(amq, torch, dev))
     return out
+
+
+def paper_form_line(amq, torch, dev):
+    """The hidden-1024 LSTM in the paper's own form (separate W_i / W_h, inputs = rows of a quantized embedding,
+    only h quantized on-line), 3/3/3 bits, 64 sequences, 35 timesteps: input projections of all timesteps in
+    one batched product, then quantize(h) + product with W_h per timestep."""
+    I = H = 1024
+    k_w = k_e = k_a = 3
+    batch, steps, vocab = 64, 35, 4096
+    g = torch.Generator(device=dev)
+    g.manual_seed(2)
+    Wic, Wia = amq.quantize(torch.randn((4 * H, I), device=dev, generator=g) * 0.03, k_w, 2)
+    Whc, Wha = amq.quantize(torch.randn((4 * H, H), device=dev, generator=g) * 0.03, k_w, 2)
+    Wec, Wea = amq.quantize(torch.randn((vocab, I), device=dev, generator=g) * 0.5, k_e, 2)
+    tokens = torch.randint(0, vocab, (steps, batch), dtype=torch.int32, device=dev, generator=g)
+    h0 = torch.zeros((batch, H), device=dev)
+    c0 = torch.zeros((batch, H), device=dev)
+    h_last, c_last = torch.empty_like(h0), torch.empty_like(c0)
+    ws = amq.new_paper_workspace(H, batch, steps, k_a)
+
+    def run():
+        xc, xb = amq.embedding_rows(Wec, Wea, I, tokens)
+        amq.lstm_sequence_paper(Wic, Wia, Whc, Wha, None, I, H, xc, xb, h0, c0, k_a, 2, ws, h_last=h_last, c_last=c_last)
+
+    ms = _burst_ms(torch, run, 10)
+    return {"workload": "paper-form LSTM sequence, I=H=1024, 3/3/3 bits, %d sequences x %d timesteps (embedding gather + "
+                        "one batched input projection + per-step quantize(h) and W_h product)" % (batch, steps),
+            "ms": ms, "bound": "tensor+latency", "us_per_timestep": 1e3 * ms / steps,
+            "timesteps_per_s": batch * steps / (ms * 1e-3)}
 
 
 def cpu_baseline(wl, unit):
