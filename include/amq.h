@@ -248,6 +248,16 @@ AMQ_API amq_status amq_lstm_sequence_paper(const uint32_t* Wi_codes, const float
                                    void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Output layer of Eq. 6, y_t = softmax(W_s h_t + b_s), on logits produced by amq_binary_gemm:
+ *   logp[r][t] = logits[r][t] - log(sum_u exp(logits[r][u]))   (computed with the row maximum subtracted),
+ *   argmax[r]  = index of the largest logit of row r (the smallest index among equal maxima).
+ * logits [rows][ld] fp32, ld >= n; logp [rows][ldp] fp32 out or NULL; argmax [rows] int32 out or NULL.
+ * argmax may be the `tokens` buffer of the next amq_embedding_rows call (greedy decoding without a host round trip).
+ */
+AMQ_API amq_status amq_log_softmax_argmax(const float* logits, int rows, int n, int ld,
+                                  float* logp, int ldp, int32_t* argmax, void* stream);
+
+/*
  * The sequence calls with HOST activations and results: x_seq, h0, c0 are read from host memory
  * (pinned memory makes the copies asynchronous) into `staging`, the sequence runs, and h_last / c_last
  * (and h_seq when not NULL) are copied back to host memory; the call returns after the stream has

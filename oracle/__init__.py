@@ -51,6 +51,7 @@ _lstm = _sig("amq_oracle_lstm_step", None, _u32p, _dp, _dp, _int, _int, _int, _d
              _dp, _dp)
 _lstm_paper = _sig("amq_oracle_lstm_step_paper", None, _u32p, _dp, _u32p, _dp, _dp, _int, _int, _int, _u32p, _dp, _int,
                    _dp, _dp, _int, _int, _int, _dp, _dp)
+_lsm = _sig("amq_oracle_log_softmax_argmax", None, _dp, _int, _int, _dp, _i32p)
 _gru = _sig("amq_oracle_gru_step", None, _u32p, _dp, _dp, _int, _int, _int, _dp, _dp, _int, _int, _int, _dp)
 _lstm_seq = _sig("amq_oracle_lstm_sequence", None, _u32p, _dp, _dp, _int, _int, _int, _dp, _int, _dp, _dp,
                  _int, _int, _int, _dp, _dp, _dp)
@@ -230,6 +231,16 @@ def lstm_step_paper(Wi_codes, Wi_alpha, Wh_codes, Wh_alpha, bias, I, H, xcodes, 
     _lstm_paper(_p(Wic, _u32p), _p(Wia, _dp), _p(Whc, _u32p), _p(Wha, _dp), _p(bias, _dp), I, H, k_w,
                 _p(xc, _u32p), _p(xb, _dp), k_e, _p(h, _dp), _p(c, _dp), batch, k_a, T, _p(h_out, _dp), _p(c_out, _dp))
     return h_out, c_out
+
+
+def log_softmax_argmax(z):
+    """(rows, n) logits -> (log-probabilities (rows, n) float64, argmax (rows,) int32)."""
+    z = _d(z)
+    rows, n = z.shape
+    logp = np.zeros((rows, n))
+    arg = np.zeros(rows, dtype=np.int32)
+    _lsm(_p(z, _dp), rows, n, _p(logp, _dp), _p(arg, _i32p))
+    return logp, arg
 
 
 def gru_step(Wcodes, Walpha, bias, I, H, x, h, k_a, T):

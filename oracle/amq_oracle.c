@@ -433,6 +433,26 @@ void amq_oracle_gru_step(const uint32_t* Wcodes, const double* Walpha, const dou
     free(z); free(px); free(ph); free(zc);
 }
 
+/* ---------------------------------------------------------------------------------------------
+ * Output layer of Eq. 6: y = softmax(W_s h + b_s), stated here on given logits: log-probabilities
+ * logp[t] = z[t] - max - log(sum_u exp(z[u] - max)) and the index of the largest logit (the first
+ * one among equal maxima).  Plain definition, fp64.
+ * ------------------------------------------------------------------------------------------- */
+void amq_oracle_log_softmax_argmax(const double* z, int rows, int n, double* logp, int32_t* arg)
+{
+    for (int r = 0; r < rows; ++r) {
+        const double* zr = z + (size_t)r * n;
+        double mx = zr[0];
+        int am = 0;
+        for (int t = 1; t < n; ++t) if (zr[t] > mx) { mx = zr[t]; am = t; }
+        double sum = 0.0;
+        for (int t = 0; t < n; ++t) sum += exp(zr[t] - mx);
+        double lse = mx + log(sum);
+        for (int t = 0; t < n; ++t) logp[(size_t)r * n + t] = zr[t] - lse;
+        arg[r] = am;
+    }
+}
+
 /* Sequences: `steps` applications of the step above, from (h0, c0); x_seq is [steps][batch][I].
  * h_seq (may be NULL) receives every h_t as [steps][batch][H]. */
 void amq_oracle_lstm_sequence(const uint32_t* Wcodes, const double* Walpha, const double* bias,

@@ -52,6 +52,7 @@ EXPORTS = {
     "amq_gru_sequence_host": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _int, _vp, _int, _int, _int,
                                      _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
     "amq_workspace_status": (_int, [_vp, _vp]),
+    "amq_log_softmax_argmax": (_int, [_vp, _int, _int, _int, _vp, _int, _vp, _vp]),
     "amq_embedding_rows": (_int, [_vp, _vp, _int, _int, _int, _vp, _int, _vp, _vp, _vp]),
     "amq_lstm_paper_workspace_bytes": (_sz, [_int, _int, _int, _int]),
     "amq_lstm_step_paper": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _int, _int, _vp, _vp, _int, _vp, _vp, _int, _int, _int,
@@ -333,3 +334,14 @@ def lstm_sequence_paper(Wi_codes, Wi_alpha, Wh_codes, Wh_alpha, bias, I, H, xcod
                                         _ptr(h_seq), _ptr(h_last), _ptr(c_last), _ptr(workspace), workspace.numel(),
                                         _stream()))
     return h_seq, h_last, c_last
+
+
+def log_softmax_argmax(logits, want_logp=True, argmax=None):
+    """logits (rows, n) fp32 -> (log-probabilities (rows, n) or None, argmax (rows,) int32)."""
+    logits = _dev(logits, torch.float32, "logits")
+    rows, n = logits.shape
+    logp = torch.empty_like(logits) if want_logp else None
+    argmax = torch.empty((rows,), dtype=torch.int32, device=logits.device) if argmax is None else argmax
+    _check(_lib.amq_log_softmax_argmax(_ptr(logits), rows, n, logits.stride(0) if rows > 1 else n, _ptr(logp), n,
+                                       _ptr(argmax), _stream()))
+    return logp, argmax

@@ -81,3 +81,55 @@ def test_paper_form_sequence_and_steps(amq, I, H, kw, ke, ka, batch, steps):
     drift = np.abs(g_last.cpu().numpy() - h).max()
     print("free-running max |dh| after %d steps: %.3g" % (steps, drift))
     assert drift <= 0.05
+
+
+@pytest.mark.parametrize("rows,n", [(1, 42000), (7, 1000), (3, 33), (2, 1)])
+def test_log_softmax_argmax(amq, rows, n):
+    z = synth.normal((rows, n), 3.0, 95 + n, 1)
+    if n > 400:
+        z[0, 17] = z[0, 400] = z[0].max() + 1.0                 # equal maxima: the first index wins
+    logp, arg = amq.log_softmax_argmax(dev(z))
+    ref, rarg = oracle.log_softmax_argmax(z.astype(np.float64))
+    assert np.abs(logp.cpu().numpy() - ref).max() <= 2e-5       # fp32 sum of up to 42000 exponentials + one log
+    assert np.array_equal(arg.cpu().numpy(), rarg)
+
+
+def test_output_layer_at_vocabulary_scale_and_greedy_decoding(amq):
+    """Text8-scale language-model step (Eq. 6 end to end): embedding row -> cell -> 42000 x 1024 output product
+    -> log-softmax / arg-max, and the arg-max fed back as the next token without leaving the device."""
+    I = H = 1024
+    V, kw, ke, ka = 42000, 2, 2, 2
+    (Wic, Wia), (Whc, Wha), _, bias = model(I, H, 8, kw, ke, 97)
+    Wsc, Wsa = oracle.quantize_rows(synth.normal((V, H), 0.05, 97, 7).astype(np.float64), kw, 2)
+    Wec, Wea = oracle.quantize_rows(synth.normal((V, I), 0.5, 97, 8).astype(np.float64), ke, 2)
+    bs = synth.normal((V,), 0.1, 97, 9)
+    d = dict(Wic=cdev(Wic), Wia=dev(Wia), Whc=cdev(Whc), Wha=dev(Wha), bias=dev(bias), Wsc=cdev(Wsc), Wsa=dev(Wsa),
+             bs=dev(bs), Wec=cdev(Wec), Wea=dev(Wea))
+    ws = amq.new_paper_workspace(H, 1, 1, ka)
+    tokens = torch.tensor([1234], dtype=torch.int32, device="cuda")
+    h, c = torch.zeros((1, H), device="cuda"), torch.zeros((1, H), device="cuda")
+    ho, co = np.zeros((1, H)), np.zeros((1, H))
+    tok_o = 1234
+    for step in range(3):
+        xc, xb = amq.embedding_rows(d["Wec"], d["Wea"], I, tokens)
+        h, c = amq.lstm_step_paper(d["Wic"], d["Wia"], d["Whc"], d["Wha"], d["bias"], I, H, xc, xb, h, c, ka, 2, ws)
+        hc, hb = amq.quantize(h, ka, 2)
+        logits = amq.binary_gemm(d["Wsc"], d["Wsa"], hc, hb, H, bias=d["bs"])
+        logp, tokens = amq.log_softmax_argmax(logits)
+        # oracle, teacher-forced on the library's state of the previous step
+        ho, co = oracle.lstm_step_paper(Wic, Wia, Whc, Wha, bias, I, H, Wec[[tok_o]], Wea[[tok_o]], ho, co, ka, 2)
+        assert np.abs(h.cpu().numpy() - ho).max() <= 1e-3
+        hc_o, hb_o = oracle.quantize_rows(ho, ka, 2)
+        z_o = oracle.binary_gemm(Wsc, Wsa, hc_o, hb_o, H, bs.astype(np.float64))
+        tol = parity.output_tolerance(Wsa, hb_o, H).max()
+        assert np.abs(logits.cpu().numpy() - z_o).max() <= tol
+        lp_o, arg_o = oracle.log_softmax_argmax(z_o)
+        assert np.abs(logp.cpu().numpy() - lp_o).max() <= 2 * tol + 2e-5
+        top2 = np.sort(z_o[0])[-2:]
+        tok_g = int(tokens.cpu()[0])
+        if top2[1] - top2[0] > 2 * tol:                         # the decision is unique within the tolerance
+            assert tok_g == int(arg_o[0])
+        else:
+            assert z_o[0, tok_g] >= top2[1] - 2 * tol           # otherwise any near-maximal token is valid
+        tok_o = tok_g                                           # follow the library's choice
+        ho, co = h.cpu().numpy().astype(np.float64), c.cpu().numpy().astype(np.float64)

@@ -256,3 +256,16 @@ def test_paper_form_lstm_step_reduces_to_full_precision_when_two_bits_are_exact(
     h_out, c_out = oracle.lstm_step_paper(Wic, Wia, Whc, Wha, None, I, H, xc, xb, h, c, 2, 2)
     h_ref, c_ref = textbook_lstm(np.concatenate([Wi, Wh], axis=1), None, x, h, c, H)
     assert np.allclose(h_out, h_ref, atol=1e-12) and np.allclose(c_out, c_ref, atol=1e-12)
+
+
+def test_log_softmax_argmax_against_library_routine_and_invariants():
+    from scipy.special import log_softmax
+    z = synth.normal((5, 1000), 3.0, 23, 1).astype(np.float64)
+    z[1, 17] = z[1, 400] = z[1].max() + 1.0                     # equal maxima: the first index wins
+    z[2] += 800.0                                               # large offsets must not overflow
+    logp, arg = oracle.log_softmax_argmax(z)
+    assert np.allclose(logp, log_softmax(z, axis=1), rtol=1e-12, atol=1e-12)
+    assert np.allclose(np.exp(logp).sum(axis=1), 1.0, atol=1e-12)
+    assert np.array_equal(arg, z.argmax(axis=1)) and arg[1] == 17
+    shifted, _ = oracle.log_softmax_argmax(z + 5.0)             # invariant to a common shift
+    assert np.allclose(shifted, logp, atol=1e-10)
