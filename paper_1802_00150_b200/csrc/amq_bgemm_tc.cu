@@ -130,6 +130,14 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16])
         : "r"(taddr) : "memory");
 }
 
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, int (&v)[8])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+        : "r"(taddr) : "memory");
+}
+
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w)
 {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" :: "r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
@@ -175,6 +183,9 @@ bgemm_tc_kernel(TcParams p)
     uint64_t* done_bar = empty_bar + MAX_STAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done_bar + 1);
     volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* sAlpha = reinterpret_cast<float*>(tmem_slot + 6);        // [MT][128] coefficient of each weight plane-row (16-byte aligned)
+    float* sBeta = sAlpha + 2 * TILE_M;                             // [TB][KA]  coefficients of the activation tile
+    float* sBsum = sBeta + 256;                                     // [TB]      their sum per batch entry
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
@@ -206,18 +217,33 @@ bgemm_tc_kernel(TcParams p)
         uint32_t dst0;                                              // shared address of the row in stage 0
         if (r_all < MT * TILE_M) {
             const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
+            size_t prow = 0;                                        // plane-row index in Wcodes / Walpha
             if (r < TMp) {
                 const int l = r / k_w, i = r - l * k_w;
                 const int u = u0 + mt * p.UT + l / p.gates, gate = l % p.gates;
-                if (u < p.units)
-                    src = reinterpret_cast<const uint4*>(a.Wcodes + (((size_t)gate * p.units + u) * k_w + i) * p.wpr);
+                if (u < p.units) {
+                    prow = ((size_t)gate * p.units + u) * k_w + i;
+                    src = reinterpret_cast<const uint4*>(a.Wcodes + prow * p.wpr);
+                }
             }
             dst0 = smem_u32(stage_base) + r_all * 128;
+            // the row's coefficient, for the epilogue (its latency hides behind the main loop)
+            if (grp == 0) sAlpha[r_all] = (src && a.epilogue != EPI_DOTS) ? __ldg(a.Walpha + prow) : 0.0f;
         } else {
             const int r = r_all - MT * TILE_M;
             const int b = b0 + r / KA, j = r % KA;
-            if (r < n_mma && b < a.batch) src = reinterpret_cast<const uint4*>(a.xcodes + ((size_t)b * KA + j) * p.wpr);
+            const bool valid = r < n_mma && b < a.batch;
+            if (valid) src = reinterpret_cast<const uint4*>(a.xcodes + ((size_t)b * KA + j) * p.wpr);
             dst0 = smem_u32(stage_base) + a_stage_bytes + r * 128;
+            if (grp == 0 && r < n_mma) {
+                const bool use = valid && a.epilogue != EPI_DOTS;
+                sBeta[r] = use ? __ldg(a.xbeta + (size_t)b * KA + j) : 0.0f;
+                if (j == 0) {
+                    float sum = 0.0f;
+                    for (int jj = 0; jj < KA; ++jj) sum += use ? __ldg(a.xbeta + (size_t)b * KA + jj) : 0.0f;
+                    sBsum[r / KA] = sum;
+                }
+            }
         }
         const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
         uint32_t off[8];                                            // swizzled position of chunk j: j xor (row mod 8)
@@ -304,13 +330,7 @@ bgemm_tc_kernel(TcParams p)
     // thread = plane-row (lane of tensor memory).  Columns arrive 16 at a time; entry e of a block of 16
     // batch entries owns columns e * KA .. e * KA + KA - 1 of the block's 16 * KA columns.
     float* Yt = reinterpret_cast<float*>(smem_raw);                 // [MT][nseg][128][TB + 1], reuses the stage buffers
-    float* sBeta = Yt + (size_t)MT * p.nseg * TILE_M * (p.TB + 1);  // [TB][KA]
     const int ldy = p.TB + 1;
-    for (int idx = tid; idx < p.TB * KA; idx += nthreads) {
-        const int b = b0 + idx / KA;
-        sBeta[idx] = (b < a.batch && a.epilogue != EPI_DOTS) ? __ldg(a.xbeta + (size_t)b * KA + idx % KA) : 0.0f;
-    }
-    __syncthreads();
     // every group of four warps covers the 128 lanes once (warp w reads lane quarter w & 3); the work items
     // (M tile, column segment, block of 16 batch entries) are dealt out to those groups in turn
     const int epi_slots = mma_warp >> 2;                            // whole groups of four warps among the expanders
@@ -318,39 +338,48 @@ bgemm_tc_kernel(TcParams p)
         const int pr = (warp & 3) * 32 + lane;
         const int slot = warp >> 2;
         const int pad = p.wpr * 32 - a.n;                           // pad positions, all in the last segment
-        const int groups = p.TB >> 4;
+        const int groups = p.TB >> 3;                               // work item: 8 batch entries = 8 * KA columns
         const int l = pr / k_w, i = pr - l * k_w;
         const int gate = l % p.gates;
         const int items1 = MT * p.nseg * groups;
         for (int item = slot; item < items1; item += epi_slots) {
             const int g = item % groups, ms = item / groups;        // ms = mt * nseg + seg
             const int mt = ms / p.nseg, seg = ms - mt * p.nseg;
-            const int u = u0 + mt * p.UT + l / p.gates;
-            const bool row_ok = pr < TMp && u < p.units;
-            const size_t row = (size_t)gate * p.units + u;
-            const float alpha = (row_ok && a.epilogue != EPI_DOTS) ? __ldg(a.Walpha + row * k_w + i) : 0.0f;
             const int corr = (seg == p.nseg - 1) ? pad : 0;
-            float* yrow = Yt + ((size_t)ms * TILE_M + pr) * ldy;
-            const uint32_t tbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(ms * n_mma);
-            float y = 0.0f;
+            const uint32_t tbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(ms * n_mma + g * KA * 8);
+            int acc[KA][8];
 #pragma unroll
-            for (int c = 0; c < KA; ++c) {
-                int acc[16];
-                tmem_ld16(tbase + (uint32_t)((g * KA + c) * 16), acc);
+            for (int c = 0; c < KA; ++c) tmem_ld8(tbase + (uint32_t)(c * 8), acc[c]);
+            if (a.epilogue == EPI_DOTS) {
+                const int u = u0 + mt * p.UT + l / p.gates;
+                const bool row_ok = pr < TMp && u < p.units;
+                const size_t row = (size_t)gate * p.units + u;
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    const int col = c * 16 + k, e = col / KA, j = col % KA;      // compile-time
-                    const int bb = g * 16 + e;
-                    const int D = (acc[k] >> 12) - corr;
-                    if (a.epilogue == EPI_DOTS) {
-                        const int b = b0 + bb;
-                        if (row_ok && b < a.batch) a.D[(((size_t)b * a.m + row) * k_w + i) * KA + j] = D;
-                    } else {
-                        y += sBeta[bb * KA + j] * small_int_to_float(D);
-                        if (j == KA - 1) { yrow[bb] = alpha * y; y = 0.0f; }
-                    }
+                for (int col = 0; col < 8 * KA; ++col) {
+                    const int b = b0 + g * 8 + col / KA;
+                    if (row_ok && b < a.batch)
+                        a.D[(((size_t)b * a.m + row) * k_w + i) * KA + col % KA] = (acc[col / 8][col % 8] >> 12) - corr;
                 }
+                continue;
+            }
+            // y = alpha_i * sum_j beta_j * D_j with D_j = accumulator / 4096 - corr: the correction is taken once per
+            // batch entry, -corr * sum_j beta_j, instead of once per accumulator
+            const float alpha = sAlpha[mt * TILE_M + pr];
+            const float fcorr = -(float)corr;
+            const float* beta = sBeta + g * 8 * KA;                 // the same addresses in every lane: broadcast reads
+            const float* bsum = sBsum + g * 8;
+            float* yrow = Yt + ((size_t)ms * TILE_M + pr) * ldy + g * 8;
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                float y = fcorr * bsum[e];
+#pragma unroll
+                for (int j = 0; j < KA; ++j) {
+                    const int col = e * KA + j;
+                    y += beta[col] * small_int_to_float(acc[col / 8][col % 8] >> 12);
+                }
+                yrow[e] = alpha * y;
             }
         }
     }
@@ -475,7 +504,7 @@ bool plan(const GemmArgs& a, TcPlan* out)
     if (cols > 512) return false;
     p.tmem_cols = cols;
     const size_t stage = (size_t)128 * (p.MT * TILE_M + p.n_mma);
-    const size_t epi = ((size_t)p.MT * p.nseg * TILE_M * (p.TB + 1) + (size_t)p.TB * a.k_a) * 4;
+    const size_t epi = (size_t)p.MT * p.nseg * TILE_M * (p.TB + 1) * 4;
     int S = (int)((220 * 1024) / stage);
     if (S > MAX_STAGES) S = MAX_STAGES;
     if (S < 2) return false;
@@ -487,7 +516,7 @@ bool plan(const GemmArgs& a, TcPlan* out)
     p.mask_sign = 0x80808080u;
     p.mask_half = 0x40404040u;
     out->p = p;
-    out->smem = S * stage + (2 * MAX_STAGES + 1) * 8 + 16;
+    out->smem = S * stage + (2 * MAX_STAGES + 1) * 8 + 24 + (2 * TILE_M + 256 + 128) * 4;   // stages, barriers, slot, coefficients
     out->grid = dim3((unsigned)((mtiles + p.MT - 1) / p.MT), (unsigned)btiles);
     return out->grid.y <= 65535u && out->smem <= 227 * 1024;
 }
