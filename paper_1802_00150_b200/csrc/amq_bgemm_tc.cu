@@ -56,6 +56,12 @@ struct TcParams {
     int nstages;    // pipeline depth
     int expanders;  // operand rows of a stage, MT * 128 + n_mma, rounded up to whole warps
     int groups;     // expander groups (1 or 2) that take the pipeline steps in turn, `expanders` threads each
+    // persistent form only: a CTA walks over tiles blockIdx.x, blockIdx.x + gridDim.x, ..
+    int ntiles;     // tiles of the problem = mgroups * (tiles along the batch)
+    int mgroups;    // groups of MT M tiles
+    int nbuf;       // accumulator buffers in tensor memory (2: the epilogue of a tile overlaps the MMAs of the next)
+    int epi_warps;  // warps that only run epilogues (4 or 8)
+    int yt_bytes;   // shared memory of the epilogue's staging array
     // run-time copies of compile-time constants: the shifts of the expansion as multipliers (so that they
     // issue on the FMA pipe) and its two byte masks (so that one LOP3 takes both from registers)
     uint32_t mul[8];
@@ -98,6 +104,36 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity)
         if (mbar_try_wait(bar, parity)) return true;
     }
     return false;
+}
+
+// the same, giving up early once another role of the CTA has recorded a failure
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* failed)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    for (unsigned i = 0; i < WAIT_LIMIT && !*failed; ++i) {
+        __nanosleep(40);
+        if (mbar_try_wait(bar, parity)) return true;
+    }
+    return false;
+}
+
+// barrier 1 joins the epilogue warps only (barrier 0 is the CTA-wide one)
+__device__ __forceinline__ void epi_bar(int nthreads)
+{
+    asm volatile("bar.sync 1, %0;" :: "r"(nthreads) : "memory");
+}
+
+// the same with an OR over a per-thread flag, so that all of them take the same way out
+__device__ __forceinline__ bool epi_bar_or(int nthreads, bool flag)
+{
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 1, %2, p;\n\t"
+        "selp.b32 %0, 1, 0, q;\n\t}"
+        : "=r"(out) : "r"((uint32_t)flag), "r"(nthreads) : "memory");
+    return out != 0;
 }
 
 // K-major, 128-byte swizzle: start address (the tile base is 1024-byte aligned), leading byte offset unused (1),
@@ -157,241 +193,106 @@ __device__ __forceinline__ float small_int_to_float(int v)
     return __int_as_float(v + 0x4B400000) - 12582912.0f;
 }
 
+// one 128-bit chunk of a packed row -> its 128 operand bytes (eight 16-byte pieces at the swizzled offsets `off`)
+__device__ __forceinline__ void expand_chunk(uint32_t base, const uint32_t (&off)[8], const uint4& v, const uint32_t (&mul)[7],
+                                             uint32_t m_sign, uint32_t m_half)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t y[8];
+#pragma unroll
+        for (int s = 0; s < 7; ++s) y[s] = and_xor(w[q] * mul[s], m_sign, m_half);     // w << (7 - s)
+        y[7] = and_xor(w[q], m_sign, m_half);
+        st_shared_v4(base + off[2 * q], y[0], y[1], y[2], y[3]);
+        st_shared_v4(base + off[2 * q + 1], y[4], y[5], y[6], y[7]);
+    }
+}
+
 __device__ __forceinline__ float logistic(float v) { return 1.0f / (1.0f + __expf(-v)); }
 
+// Epilogue, first half: tensor memory -> registers -> partial products y[plane-row][batch entry] in shared memory
+// (EPI_DOTS: the integer partials straight to global memory).  A thread is a plane-row (lane of tensor memory, lane
+// quarter `quarter` = warp index mod 4); the work items (M tile, column segment, 8 batch entries = 8 * KA columns)
+// are dealt out to `nslots` groups of four warps.  Reads of the accumulators are complete on return.
 template <int KA>
-__global__ void __launch_bounds__(MAX_THREADS, 1)
-bgemm_tc_kernel(TcParams p)
+__device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_t tmem_acc, int u0, int b0, int quarter, int lane,
+                                                      int slot, int nslots, const float* sAlpha, const float* sBeta,
+                                                      const float* sBcorr, float* Yt)
 {
-    extern __shared__ __align__(1024) unsigned char smem_raw[];
     const GemmArgs& a = p.a;
-    const int k_w = a.k_w;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int TM = p.UT * p.gates;                  // weight rows of an M tile
-    const int TMp = TM * k_w;                       // plane-rows in use per M tile (<= 128)
-    const int MT = p.MT, S = p.nstages, G = p.groups;
-    const int EXP = p.expanders;                    // operand rows rounded up to whole warps
-    const int mma_warp = (G * EXP) >> 5, nthreads = G * EXP + 32;
-    const int n_mma = p.n_mma;
-    const int a_stage_bytes = MT * TILE_M * 128;    // 128 bytes of K per row and stage
-    const int stage_bytes = a_stage_bytes + n_mma * 128;
-    const int u0 = blockIdx.x * p.UT * MT, b0 = blockIdx.y * p.TB;
-
-    unsigned char* stage_base = smem_raw;
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)S * stage_bytes);   // [S]
-    uint64_t* empty_bar = full_bar + MAX_STAGES;                                            // [S]
-    uint64_t* done_bar = empty_bar + MAX_STAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done_bar + 1);
-    volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    float* sAlpha = reinterpret_cast<float*>(tmem_slot + 6);        // [MT][128] coefficient of each weight plane-row (16-byte aligned)
-    float* sBeta = sAlpha + 2 * TILE_M;                             // [TB][KA]  coefficients of the activation tile
-    float* sBsum = sBeta + 256;                                     // [TB]      their sum per batch entry
-
-    if (tid == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(smem_u32(&full_bar[s]), (uint32_t)EXP);
-            mbar_init(smem_u32(&empty_bar[s]), 1);
-        }
-        mbar_init(smem_u32(done_bar), 1);
-        *failed = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == mma_warp) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem_base = *tmem_slot;
-
-    const int CH = p.wpr >> 2;                                      // 128-bit chunks along K = pipeline steps
-    const int split_word = (p.nseg == 2) ? (a.I >> 5) : p.wpr;      // first word of the second column segment
-
-    if (warp < mma_warp) {
-        // ---- expanders: G groups of EXP threads take the steps in turn; inside a group thread r owns operand
-        //      row r (A plane-rows first, then the B rows) ----
-        const int grp = tid / EXP, r_all = tid - grp * EXP;
-        const uint4* src = nullptr;
-        uint32_t dst0;                                              // shared address of the row in stage 0
-        if (r_all < MT * TILE_M) {
-            const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
-            size_t prow = 0;                                        // plane-row index in Wcodes / Walpha
-            if (r < TMp) {
-                const int l = r / k_w, i = r - l * k_w;
-                const int u = u0 + mt * p.UT + l / p.gates, gate = l % p.gates;
-                if (u < p.units) {
-                    prow = ((size_t)gate * p.units + u) * k_w + i;
-                    src = reinterpret_cast<const uint4*>(a.Wcodes + prow * p.wpr);
-                }
-            }
-            dst0 = smem_u32(stage_base) + r_all * 128;
-            // the row's coefficient, for the epilogue (its latency hides behind the main loop)
-            if (grp == 0) sAlpha[r_all] = (src && a.epilogue != EPI_DOTS) ? __ldg(a.Walpha + prow) : 0.0f;
-        } else {
-            const int r = r_all - MT * TILE_M;
-            const int b = b0 + r / KA, j = r % KA;
-            const bool valid = r < n_mma && b < a.batch;
-            if (valid) src = reinterpret_cast<const uint4*>(a.xcodes + ((size_t)b * KA + j) * p.wpr);
-            dst0 = smem_u32(stage_base) + a_stage_bytes + r * 128;
-            if (grp == 0 && r < n_mma) {
-                const bool use = valid && a.epilogue != EPI_DOTS;
-                sBeta[r] = use ? __ldg(a.xbeta + (size_t)b * KA + j) : 0.0f;
-                if (j == 0) {
-                    float sum = 0.0f;
-                    for (int jj = 0; jj < KA; ++jj) sum += use ? __ldg(a.xbeta + (size_t)b * KA + jj) : 0.0f;
-                    sBsum[r / KA] = sum;
-                }
-            }
-        }
-        const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
-        uint32_t off[8];                                            // swizzled position of chunk j: j xor (row mod 8)
-#pragma unroll
-        for (int j = 0; j < 8; ++j) off[j] = (uint32_t)((j ^ (r_all & 7)) << 4);
-        uint32_t mul[7];
-#pragma unroll
-        for (int s = 0; s < 7; ++s) mul[s] = p.mul[s];
-        const uint32_t m_sign = p.mask_sign, m_half = p.mask_half;  // 0x80808080, 0x40404040
-        const uint4 zero = make_uint4(0, 0, 0, 0);
-
-        uint4 cur = (src && grp < CH) ? __ldg(src + grp) : zero;    // own steps: grp, grp + G, ..
-        uint4 nxt = (src && grp + G < CH) ? __ldg(src + grp + G) : zero;
-        int buf = grp;                                              // G <= S
-        uint32_t empty_parity = 1;                                  // parity that means "never used" on the first lap
-        for (int c = grp; c < CH; c += G) {
-            const uint4 v = cur;
-            cur = nxt;
-            nxt = (src && c + 2 * G < CH) ? __ldg(src + c + 2 * G) : zero;
-            // the MMAs that read this buffer one lap ago must have completed
-            if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; break; }
-            if (writes) {
-                const uint32_t base = dst0 + (uint32_t)(buf * stage_bytes);
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint32_t y[8];
-#pragma unroll
-                    for (int s = 0; s < 7; ++s) y[s] = and_xor(w[q] * mul[s], m_sign, m_half);     // w << (7 - s)
-                    y[7] = and_xor(w[q], m_sign, m_half);
-                    st_shared_v4(base + off[2 * q], y[0], y[1], y[2], y[3]);
-                    st_shared_v4(base + off[2 * q + 1], y[4], y[5], y[6], y[7]);
-                }
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
-            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
-            buf += G;
-            if (buf >= S) { buf -= S; empty_parity ^= 1u; }
-        }
-    } else if (lane == 0) {
-        // ---- MMA issuer ----
-        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
-        const uint64_t desc_base = smem_desc(smem_u32(stage_base)); // descriptor of stage 0, tile 0, word 0
-        int buf = 0;
-        uint32_t full_parity = 0;
-        for (int c = 0; c < CH; ++c) {
-            if (!mbar_wait(smem_u32(&full_bar[buf]), full_parity)) { *failed = 1; break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // descriptors of the stage: start addresses are below 256 KiB, so adding to the low word never carries
-            const uint64_t adesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
-            const uint64_t bdesc0 = adesc0 + (uint64_t)(a_stage_bytes >> 4);
-#pragma unroll
-            for (int qq = 0; qq < STAGE_WORDS; ++qq) {
-                const int word = c * STAGE_WORDS + qq;
-                const int seg = word >= split_word ? 1 : 0;
-                const uint32_t accumulate = (word != 0 && word != split_word) ? 1u : 0u;
-                mma_i8(tmem_base + seg * n_mma, adesc0 + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
-                if (MT == 2)
-                    mma_i8(tmem_base + (p.nseg + seg) * n_mma, adesc0 + (TILE_M * 128 >> 4) + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
-            }
-            mma_commit(smem_u32(&empty_bar[buf]));
-            if (++buf == S) { buf = 0; full_parity ^= 1u; }
-        }
-        if (!*failed) mma_commit(smem_u32(done_bar));               // covers every MMA issued above
-    }
-    __syncwarp();
-
-    // all MMAs done?
-    bool ok = !*failed;
-    if (ok) ok = mbar_wait_relaxed(smem_u32(done_bar), 0);
-    if (__syncthreads_or(!ok)) {
-        // give the tensor core time to drain what was issued, then release tensor memory and leave
-        if (tid == 0) atomicExch(&g_tc_status, 1u);
-        __nanosleep(1000000);
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
-        if (warp == mma_warp)
-            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
-        return;
-    }
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-
-    // ---- epilogue 1: tensor memory -> registers -> partial products in shared memory ----
-    // thread = plane-row (lane of tensor memory).  Columns arrive 16 at a time; entry e of a block of 16
-    // batch entries owns columns e * KA .. e * KA + KA - 1 of the block's 16 * KA columns.
-    float* Yt = reinterpret_cast<float*>(smem_raw);                 // [MT][nseg][128][TB + 1], reuses the stage buffers
-    const int ldy = p.TB + 1;
-    // every group of four warps covers the 128 lanes once (warp w reads lane quarter w & 3); the work items
-    // (M tile, column segment, block of 16 batch entries) are dealt out to those groups in turn
-    const int epi_slots = mma_warp >> 2;                            // whole groups of four warps among the expanders
-    if (warp < 4 * epi_slots) {
-        const int pr = (warp & 3) * 32 + lane;
-        const int slot = warp >> 2;
-        const int pad = p.wpr * 32 - a.n;                           // pad positions, all in the last segment
-        const int groups = p.TB >> 3;                               // work item: 8 batch entries = 8 * KA columns
+    const int k_w = a.k_w, n_mma = p.n_mma, ldy = p.TB + 1;
+    const int TMp = p.UT * p.gates * k_w;
+    const int pr = quarter * 32 + lane;
+    const int groups = p.TB >> 3;
+    const int items1 = p.MT * p.nseg * groups;
+    const uint32_t tlane = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+    if (a.epilogue == EPI_DOTS) {
+        const int pad = p.wpr * 32 - a.n;
         const int l = pr / k_w, i = pr - l * k_w;
         const int gate = l % p.gates;
-        const int items1 = MT * p.nseg * groups;
-        for (int item = slot; item < items1; item += epi_slots) {
-            const int g = item % groups, ms = item / groups;        // ms = mt * nseg + seg
-            const int mt = ms / p.nseg, seg = ms - mt * p.nseg;
-            const int corr = (seg == p.nseg - 1) ? pad : 0;
-            const uint32_t tbase = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(ms * n_mma + g * KA * 8);
+        for (int item = slot; item < items1; item += nslots) {
+            const int g = item % groups, mt = item / groups;        // (one column segment in this epilogue)
+            const int u = u0 + mt * p.UT + l / p.gates;
+            const bool row_ok = pr < TMp && u < p.units;
+            const size_t row = (size_t)gate * p.units + u;
             int acc[KA][8];
 #pragma unroll
-            for (int c = 0; c < KA; ++c) tmem_ld8(tbase + (uint32_t)(c * 8), acc[c]);
-            if (a.epilogue == EPI_DOTS) {
-                const int u = u0 + mt * p.UT + l / p.gates;
-                const bool row_ok = pr < TMp && u < p.units;
-                const size_t row = (size_t)gate * p.units + u;
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                for (int col = 0; col < 8 * KA; ++col) {
-                    const int b = b0 + g * 8 + col / KA;
-                    if (row_ok && b < a.batch)
-                        a.D[(((size_t)b * a.m + row) * k_w + i) * KA + col % KA] = (acc[col / 8][col % 8] >> 12) - corr;
-                }
-                continue;
-            }
-            // y = alpha_i * sum_j beta_j * D_j with D_j = accumulator / 4096 - corr: the correction is taken once per
-            // batch entry, -corr * sum_j beta_j, instead of once per accumulator
-            const float alpha = sAlpha[mt * TILE_M + pr];
-            const float fcorr = -(float)corr;
-            const float* beta = sBeta + g * 8 * KA;                 // the same addresses in every lane: broadcast reads
-            const float* bsum = sBsum + g * 8;
-            float* yrow = Yt + ((size_t)ms * TILE_M + pr) * ldy + g * 8;
+            for (int c = 0; c < KA; ++c) tmem_ld8(tlane + (uint32_t)(mt * n_mma + g * KA * 8 + c * 8), acc[c]);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                float y = fcorr * bsum[e];
+            for (int col = 0; col < 8 * KA; ++col) {
+                const int b = b0 + g * 8 + col / KA;
+                if (row_ok && b < a.batch)
+                    a.D[(((size_t)b * a.m + row) * k_w + i) * KA + col % KA] = (acc[col / 8][col % 8] >> 12) - pad;
+            }
+        }
+        return;
+    }
+    for (int item = slot; item < items1; item += nslots) {
+        const int g = item % groups, ms = item / groups;            // ms = mt * nseg + seg
+        const int mt = ms / p.nseg, seg = ms - mt * p.nseg;
+        int acc[KA][8];
+#pragma unroll
+        for (int c = 0; c < KA; ++c) tmem_ld8(tlane + (uint32_t)(ms * n_mma + g * KA * 8 + c * 8), acc[c]);
+        // y = alpha_i * sum_j beta_j * D_j with D_j = accumulator / 4096 - pad; the pad correction is taken once per
+        // batch entry (sBcorr = -pad * sum_j beta_j), in the last column segment
+        const float alpha = sAlpha[mt * TILE_M + pr];
+        const bool last = seg == p.nseg - 1;
+        float* yrow = Yt + ((size_t)ms * TILE_M + pr) * ldy + g * 8;
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            // coefficients of four entries: 4 * KA consecutive floats, 16-byte aligned
+            float4 b4[KA];
+#pragma unroll
+            for (int q = 0; q < KA; ++q) b4[q] = reinterpret_cast<const float4*>(sBeta + (g * 8 + half * 4) * KA)[q];
+            const float4 c4 = *reinterpret_cast<const float4*>(sBcorr + g * 8 + half * 4);
+            const float corr4[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+            for (int e4 = 0; e4 < 4; ++e4) {
+                float y = last ? corr4[e4] : 0.0f;
 #pragma unroll
                 for (int j = 0; j < KA; ++j) {
-                    const int col = e * KA + j;
-                    y += beta[col] * small_int_to_float(acc[col / 8][col % 8] >> 12);
+                    const int bi = e4 * KA + j;                     // index among the 4 * KA coefficients
+                    const float4 t = b4[bi >> 2];
+                    const float beta = (bi & 3) == 0 ? t.x : (bi & 3) == 1 ? t.y : (bi & 3) == 2 ? t.z : t.w;
+                    const int col = (half * 4 + e4) * KA + j;
+                    y += beta * small_int_to_float(acc[col / 8][col % 8] >> 12);
                 }
-                yrow[e] = alpha * y;
+                yrow[half * 4 + e4] = alpha * y;
             }
         }
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (warp == mma_warp)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
-    if (a.epilogue == EPI_DOTS) return;
+}
 
-    // ---- epilogue 2: sum the k_w planes of each weight row, bias, gates ----
+// Epilogue, second half: sum the k_w planes of each weight row, bias, gates; `nthreads` threads numbered `tid`.
+__device__ __forceinline__ void epilogue_smem_to_global(const TcParams& p, const float* Yt, int u0, int b0, int tid, int nthreads)
+{
     // thread -> (row or unit, every `bstep`-th batch entry): one division per thread, none per output
-    const int TB = p.TB;
+    const GemmArgs& a = p.a;
+    const int k_w = a.k_w, TB = p.TB, MT = p.MT, ldy = p.TB + 1;
+    const int TM = p.UT * p.gates;
     const int per_tile = (a.epilogue == EPI_Y) ? TM : p.UT;         // rows (plain) or units (cells) of an M tile
     const int items = MT * per_tile;
     const int lanes_b = nthreads / items;                           // threads sharing one row / unit (0: fewer threads than items)
@@ -470,11 +371,458 @@ bgemm_tc_kernel(TcParams p)
     }
 }
 
+template <int KA>
+__global__ void __launch_bounds__(MAX_THREADS, 1)
+bgemm_tc_kernel(TcParams p)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    const GemmArgs& a = p.a;
+    const int k_w = a.k_w;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int TM = p.UT * p.gates;                  // weight rows of an M tile
+    const int TMp = TM * k_w;                       // plane-rows in use per M tile (<= 128)
+    const int MT = p.MT, S = p.nstages, G = p.groups;
+    const int EXP = p.expanders;                    // operand rows rounded up to whole warps
+    const int mma_warp = (G * EXP) >> 5, nthreads = G * EXP + 32;
+    const int n_mma = p.n_mma;
+    const int a_stage_bytes = MT * TILE_M * 128;    // 128 bytes of K per row and stage
+    const int stage_bytes = a_stage_bytes + n_mma * 128;
+    const int u0 = blockIdx.x * p.UT * MT, b0 = blockIdx.y * p.TB;
+
+    unsigned char* stage_base = smem_raw;
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)S * stage_bytes);   // [S]
+    uint64_t* empty_bar = full_bar + MAX_STAGES;                                            // [S]
+    uint64_t* done_bar = empty_bar + MAX_STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(done_bar + 1);
+    volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* sAlpha = reinterpret_cast<float*>(tmem_slot + 6);        // [MT][128] coefficient of each weight plane-row (16-byte aligned)
+    float* sBeta = sAlpha + 2 * TILE_M;                             // [TB][KA]  coefficients of the activation tile
+    float* sBcorr = sBeta + 256;                                    // [TB]      -pad * their sum per batch entry
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), (uint32_t)EXP);
+            mbar_init(smem_u32(&empty_bar[s]), 1);
+        }
+        mbar_init(smem_u32(done_bar), 1);
+        *failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == mma_warp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int CH = p.wpr >> 2;                                      // 128-bit chunks along K = pipeline steps
+    const int split_word = (p.nseg == 2) ? (a.I >> 5) : p.wpr;      // first word of the second column segment
+
+    if (warp < mma_warp) {
+        // ---- expanders: G groups of EXP threads take the steps in turn; inside a group thread r owns operand
+        //      row r (A plane-rows first, then the B rows) ----
+        const int grp = tid / EXP, r_all = tid - grp * EXP;
+        const uint4* src = nullptr;
+        uint32_t dst0;                                              // shared address of the row in stage 0
+        if (r_all < MT * TILE_M) {
+            const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
+            size_t prow = 0;                                        // plane-row index in Wcodes / Walpha
+            if (r < TMp) {
+                const int l = r / k_w, i = r - l * k_w;
+                const int u = u0 + mt * p.UT + l / p.gates, gate = l % p.gates;
+                if (u < p.units) {
+                    prow = ((size_t)gate * p.units + u) * k_w + i;
+                    src = reinterpret_cast<const uint4*>(a.Wcodes + prow * p.wpr);
+                }
+            }
+            dst0 = smem_u32(stage_base) + r_all * 128;
+            // the row's coefficient, for the epilogue (its latency hides behind the main loop)
+            if (grp == 0) sAlpha[r_all] = (src && a.epilogue != EPI_DOTS) ? __ldg(a.Walpha + prow) : 0.0f;
+        } else {
+            const int r = r_all - MT * TILE_M;
+            const int b = b0 + r / KA, j = r % KA;
+            const bool valid = r < n_mma && b < a.batch;
+            if (valid) src = reinterpret_cast<const uint4*>(a.xcodes + ((size_t)b * KA + j) * p.wpr);
+            dst0 = smem_u32(stage_base) + a_stage_bytes + r * 128;
+            if (grp == 0 && r < n_mma) {
+                const bool use = valid && a.epilogue != EPI_DOTS;
+                sBeta[r] = use ? __ldg(a.xbeta + (size_t)b * KA + j) : 0.0f;
+                if (j == 0) {
+                    float sum = 0.0f;
+                    for (int jj = 0; jj < KA; ++jj) sum += use ? __ldg(a.xbeta + (size_t)b * KA + jj) : 0.0f;
+                    sBcorr[r / KA] = -(float)(p.wpr * 32 - a.n) * sum;
+                }
+            }
+        }
+        const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
+        uint32_t off[8];                                            // swizzled position of chunk j: j xor (row mod 8)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) off[j] = (uint32_t)((j ^ (r_all & 7)) << 4);
+        uint32_t mul[7];
+#pragma unroll
+        for (int s = 0; s < 7; ++s) mul[s] = p.mul[s];
+        const uint32_t m_sign = p.mask_sign, m_half = p.mask_half;  // 0x80808080, 0x40404040
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+
+        uint4 cur = (src && grp < CH) ? __ldg(src + grp) : zero;    // own steps: grp, grp + G, ..
+        uint4 nxt = (src && grp + G < CH) ? __ldg(src + grp + G) : zero;
+        int buf = grp;                                              // G <= S
+        uint32_t empty_parity = 1;                                  // parity that means "never used" on the first lap
+        for (int c = grp; c < CH; c += G) {
+            const uint4 v = cur;
+            cur = nxt;
+            nxt = (src && c + 2 * G < CH) ? __ldg(src + c + 2 * G) : zero;
+            // the MMAs that read this buffer one lap ago must have completed
+            if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; break; }
+            if (writes) {
+                expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, v, mul, m_sign, m_half);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
+            buf += G;
+            if (buf >= S) { buf -= S; empty_parity ^= 1u; }
+        }
+    } else if (lane == 0) {
+        // ---- MMA issuer ----
+        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+        const uint64_t desc_base = smem_desc(smem_u32(stage_base)); // descriptor of stage 0, tile 0, word 0
+        int buf = 0;
+        uint32_t full_parity = 0;
+        for (int c = 0; c < CH; ++c) {
+            if (!mbar_wait(smem_u32(&full_bar[buf]), full_parity)) { *failed = 1; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // descriptors of the stage: start addresses are below 256 KiB, so adding to the low word never carries
+            const uint64_t adesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
+            const uint64_t bdesc0 = adesc0 + (uint64_t)(a_stage_bytes >> 4);
+#pragma unroll
+            for (int qq = 0; qq < STAGE_WORDS; ++qq) {
+                const int word = c * STAGE_WORDS + qq;
+                const int seg = word >= split_word ? 1 : 0;
+                const uint32_t accumulate = (word != 0 && word != split_word) ? 1u : 0u;
+                mma_i8(tmem_base + seg * n_mma, adesc0 + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                if (MT == 2)
+                    mma_i8(tmem_base + (p.nseg + seg) * n_mma, adesc0 + (TILE_M * 128 >> 4) + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+            }
+            mma_commit(smem_u32(&empty_bar[buf]));
+            if (++buf == S) { buf = 0; full_parity ^= 1u; }
+        }
+        if (!*failed) mma_commit(smem_u32(done_bar));               // covers every MMA issued above
+    }
+    __syncwarp();
+
+    // all MMAs done?
+    bool ok = !*failed;
+    if (ok) ok = mbar_wait_relaxed(smem_u32(done_bar), 0);
+    if (__syncthreads_or(!ok)) {
+        // give the tensor core time to drain what was issued, then release tensor memory and leave
+        if (tid == 0) atomicExch(&g_tc_status, 1u);
+        __nanosleep(1000000);
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (warp == mma_warp)
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+        return;
+    }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+    // ---- epilogue: tensor memory -> partial products in shared memory (reusing the stage buffers) -> results ----
+    float* Yt = reinterpret_cast<float*>(smem_raw);                 // [MT][nseg][128][TB + 1]
+    const int epi_slots = mma_warp >> 2;                            // whole groups of four warps among the expanders
+    if (warp < 4 * epi_slots)
+        epilogue_tmem_to_smem<KA>(p, tmem_base, u0, b0, warp & 3, lane, warp >> 2, epi_slots, sAlpha, sBeta, sBcorr, Yt);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == mma_warp)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+    if (a.epilogue == EPI_DOTS) return;
+
+    epilogue_smem_to_global(p, Yt, u0, b0, tid, nthreads);
+}
+
+// The persistent form of the kernel, for problems of more tiles than the GPU has SMs: one CTA per SM walks over
+// tiles t = blockIdx.x, blockIdx.x + gridDim.x, ..  The accumulators are double-buffered in tensor memory and
+// dedicated warps run the epilogue, so that the epilogue of a tile (arithmetic and global stores) overlaps the
+// expansion and the MMAs of the next one (bound by shared-memory traffic).  The stage pipeline runs on across
+// tiles; "accumulator full" barriers are signalled by tcgen05.commit after the last MMA of a tile,
+// "accumulator empty" ones by the epilogue warps after their last read of tensor memory.
+template <int KA>
+__global__ void __launch_bounds__(MAX_THREADS, 1)
+bgemm_tc_persistent_kernel(TcParams p)
+{
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    const GemmArgs& a = p.a;
+    const int k_w = a.k_w;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int TMp = p.UT * p.gates * k_w;           // plane-rows in use per M tile (<= 128)
+    const int MT = p.MT, S = p.nstages, G = p.groups, EXP = p.expanders;
+    const int mma_warp = (G * EXP) >> 5, epi_warp0 = mma_warp + 1, EW = p.epi_warps;
+    const int n_mma = p.n_mma;
+    const int a_stage_bytes = MT * TILE_M * 128;
+    const int stage_bytes = a_stage_bytes + n_mma * 128;
+    const int acc_cols = MT * p.nseg * n_mma;       // columns of one accumulator buffer
+    const int CH = p.wpr >> 2;                      // pipeline steps per tile
+    const int split_word = (p.nseg == 2) ? (a.I >> 5) : p.wpr;
+    const int ntiles = p.ntiles, MG = p.mgroups, tile_step = (int)gridDim.x;
+
+    unsigned char* stage_base = smem_raw;
+    float* Yt = reinterpret_cast<float*>(smem_raw + (size_t)S * stage_bytes);               // [MT][nseg][128][TB + 1]
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)S * stage_bytes + p.yt_bytes);   // [S]
+    uint64_t* empty_bar = full_bar + MAX_STAGES;                                            // [S]
+    uint64_t* tfull_bar = empty_bar + MAX_STAGES;                                           // [2] accumulator buffer complete
+    uint64_t* tempty_bar = tfull_bar + 2;                                                   // [2] accumulator buffer read out
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+    volatile int* failed = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* sAlpha = reinterpret_cast<float*>(tmem_slot + 4);        // [MT][128]
+    float* sBeta = sAlpha + 2 * TILE_M;                             // [TB][KA]
+    float* sBcorr = sBeta + 256;                                    // [TB]
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), (uint32_t)EXP);
+            mbar_init(smem_u32(&empty_bar[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&tfull_bar[b]), 1);
+            mbar_init(smem_u32(&tempty_bar[b]), (uint32_t)EW);      // one arrival per epilogue warp
+        }
+        *failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == mma_warp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < mma_warp) {
+        // ---- expanders: thread r of a group owns operand row r of every tile; the groups take the steps of the
+        //      CTA's whole sequence (tiles x steps per tile) in turn ----
+        const int grp = tid / EXP, r_all = tid - grp * EXP;
+        const bool is_a = r_all < MT * TILE_M;
+        int unit_off = 0, gate = 0, plane = 0, entry = 0;
+        bool valid;
+        uint32_t dst0;
+        if (is_a) {
+            const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
+            const int l = r / k_w;
+            valid = r < TMp;
+            plane = r - l * k_w; unit_off = mt * p.UT + l / p.gates; gate = l % p.gates;
+            dst0 = smem_u32(stage_base) + r_all * 128;
+        } else {
+            const int r = r_all - MT * TILE_M;
+            valid = r < n_mma;
+            entry = r / KA; plane = r % KA;
+            dst0 = smem_u32(stage_base) + a_stage_bytes + r * 128;
+        }
+        const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
+        // packed row of this thread in tile `tile` (null: beyond the matrix, the batch or the CTA's last tile)
+        auto row_of = [&](int tile) -> const uint4* {
+            if (!valid || tile >= ntiles) return nullptr;
+            const int bt = tile / MG, mg = tile - bt * MG;
+            if (is_a) {
+                const int u = mg * p.UT * MT + unit_off;
+                return u < p.units ? reinterpret_cast<const uint4*>(a.Wcodes + (((size_t)gate * p.units + u) * k_w + plane) * p.wpr)
+                                   : nullptr;
+            }
+            const int b = bt * p.TB + entry;
+            return b < a.batch ? reinterpret_cast<const uint4*>(a.xcodes + ((size_t)b * KA + plane) * p.wpr) : nullptr;
+        };
+        uint32_t off[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) off[j] = (uint32_t)((j ^ (r_all & 7)) << 4);
+        uint32_t mul[7];
+#pragma unroll
+        for (int s = 0; s < 7; ++s) mul[s] = p.mul[s];
+        const uint32_t m_sign = p.mask_sign, m_half = p.mask_half;
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+
+        // load cursor: runs two of the group's steps ahead of the expansion, across tile boundaries
+        int pf_tile = (int)blockIdx.x, pf_c = grp;
+        const uint4* pf_src = row_of(pf_tile);
+        auto pf_load = [&]() -> uint4 {
+            while (pf_c >= CH) { pf_c -= CH; pf_tile += tile_step; pf_src = row_of(pf_tile); }
+            const uint4 v = pf_src ? __ldg(pf_src + pf_c) : zero;
+            pf_c += G;
+            return v;
+        };
+        const int my_tiles = (ntiles - (int)blockIdx.x + tile_step - 1) / tile_step;
+        const int total = my_tiles * CH;
+        uint4 cur = pf_load(), nxt = pf_load();
+        int buf = grp;                                              // G <= S
+        uint32_t empty_parity = 1;
+        for (int q = grp; q < total; q += G) {
+            const uint4 v = cur;
+            cur = nxt;
+            nxt = pf_load();
+            if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity, failed)) { *failed = 1; break; }
+            if (writes) expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, v, mul, m_sign, m_half);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
+            buf += G;
+            if (buf >= S) { buf -= S; empty_parity ^= 1u; }
+        }
+    } else if (warp == mma_warp) {
+        if (lane == 0) {
+            // ---- MMA issuer ----
+            const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+            const uint64_t desc_base = smem_desc(smem_u32(stage_base));
+            int buf = 0;
+            uint32_t full_parity = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = (int)blockIdx.x; tile < ntiles && ok; tile += tile_step, ++it) {
+                const int ab = (p.nbuf == 2) ? (it & 1) : 0;
+                const uint32_t use = (p.nbuf == 2) ? (uint32_t)(it >> 1) : (uint32_t)it;    // earlier uses of this buffer
+                // the epilogue of the tile that used this buffer last must have read it out
+                if (!mbar_wait(smem_u32(&tempty_bar[ab]), (use & 1u) ^ 1u)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t acc = tmem_base + (uint32_t)(ab * acc_cols);
+                for (int c = 0; c < CH; ++c) {
+                    if (!mbar_wait(smem_u32(&full_bar[buf]), full_parity)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t adesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
+                    const uint64_t bdesc0 = adesc0 + (uint64_t)(a_stage_bytes >> 4);
+#pragma unroll
+                    for (int qq = 0; qq < STAGE_WORDS; ++qq) {
+                        const int word = c * STAGE_WORDS + qq;
+                        const int seg = word >= split_word ? 1 : 0;
+                        const uint32_t accumulate = (word != 0 && word != split_word) ? 1u : 0u;
+                        mma_i8(acc + seg * n_mma, adesc0 + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                        if (MT == 2)
+                            mma_i8(acc + (p.nseg + seg) * n_mma, adesc0 + (TILE_M * 128 >> 4) + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                    }
+                    mma_commit(smem_u32(&empty_bar[buf]));
+                    if (++buf == S) { buf = 0; full_parity ^= 1u; }
+                }
+                if (ok) mma_commit(smem_u32(&tfull_bar[ab]));       // covers every MMA of the tile
+            }
+            if (!ok) *failed = 1;
+        }
+    } else {
+        // ---- epilogue warps ----
+        const int tid_e = tid - epi_warp0 * 32, nth_e = EW * 32;
+        const int quarter = warp & 3, slot = (warp - epi_warp0) >> 2, nslots = EW >> 2;
+        int it = 0;
+        for (int tile = (int)blockIdx.x; tile < ntiles; tile += tile_step, ++it) {
+            const int ab = (p.nbuf == 2) ? (it & 1) : 0;
+            const uint32_t use = (p.nbuf == 2) ? (uint32_t)(it >> 1) : (uint32_t)it;
+            const int bt = tile / MG, mg = tile - bt * MG;
+            const int u0 = mg * p.UT * MT, b0 = bt * p.TB;
+            // coefficients of the tile (every thread is past the previous tile's first half, which read the old ones)
+            if (a.epilogue != EPI_DOTS) {
+                for (int idx = tid_e; idx < MT * TILE_M; idx += nth_e) {
+                    const int mt = idx >> 7, r = idx & (TILE_M - 1);
+                    const int l = r / k_w, i = r - l * k_w;
+                    const int u = u0 + mt * p.UT + l / p.gates, gate = l % p.gates;
+                    sAlpha[idx] = (r < TMp && u < p.units) ? __ldg(a.Walpha + ((size_t)gate * p.units + u) * k_w + i) : 0.0f;
+                }
+                for (int idx = tid_e; idx < n_mma; idx += nth_e) {
+                    const int e = idx / KA, j = idx - e * KA, b = b0 + e;
+                    const bool use_b = b < a.batch;
+                    sBeta[idx] = use_b ? __ldg(a.xbeta + (size_t)b * KA + j) : 0.0f;
+                    if (j == 0) {
+                        float sum = 0.0f;
+                        for (int jj = 0; jj < KA; ++jj) sum += use_b ? __ldg(a.xbeta + (size_t)b * KA + jj) : 0.0f;
+                        sBcorr[e] = -(float)(p.wpr * 32 - a.n) * sum;
+                    }
+                }
+            }
+            const bool ok = mbar_wait_relaxed(smem_u32(&tfull_bar[ab]), use & 1u, failed);
+            __syncwarp();
+            // one barrier: the coefficients are visible, every thread has left the previous tile's second half
+            // (the staging array is free), and all threads agree on whether to go on
+            if (epi_bar_or(nth_e, !ok || *failed)) { if (!ok) *failed = 1; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            epilogue_tmem_to_smem<KA>(p, tmem_base + (uint32_t)(ab * acc_cols), u0, b0, quarter, lane, slot, nslots,
+                                      sAlpha, sBeta, sBcorr, Yt);
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0)
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&tempty_bar[ab])) : "memory");
+            if (a.epilogue == EPI_DOTS) continue;
+            __syncwarp();
+            epi_bar(nth_e);                                         // the staging array is complete
+            epilogue_smem_to_global(p, Yt, u0, b0, tid_e, nth_e);
+            __syncwarp();
+        }
+    }
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    const bool bad = __syncthreads_or(*failed != 0);
+    if (bad) {
+        // give the tensor core time to drain what was issued before tensor memory is released
+        if (tid == 0) atomicExch(&g_tc_status, 1u);
+        __nanosleep(1000000);
+        __syncthreads();
+    }
+    if (warp == mma_warp)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+}
+
 struct TcPlan {
     TcParams p;
     dim3 grid;
     size_t smem;
+    int threads;
+    bool persistent;
 };
+
+int sm_count()
+{
+    static int count = 0;       // the same on every device of a node
+    if (count == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            count = v;
+        else
+            return 148;
+    }
+    return count;
+}
+
+// The persistent form: one M tile per CTA step, two accumulator buffers, dedicated epilogue warps.  Possible when
+// both buffers fit tensor memory and there are more tiles than SMs (otherwise nothing could overlap).
+bool plan_persistent(const TcParams& base, int mtiles, int btiles, TcPlan* out)
+{
+    TcParams p = base;
+    p.MT = 1;
+    p.mgroups = mtiles;
+    const int sms = sm_count();
+    if (mtiles > 0x7fffffff / btiles) return false;
+    p.ntiles = mtiles * btiles;
+    if (p.ntiles <= sms) return false;
+    const int acc_cols = p.nseg * p.n_mma;
+    if (2 * acc_cols > 512) return false;
+    p.nbuf = 2;
+    int cols = 32;
+    while (cols < 2 * acc_cols) cols <<= 1;
+    p.tmem_cols = cols;
+    const size_t stage = (size_t)128 * (TILE_M + p.n_mma);
+    p.yt_bytes = (int)(((size_t)p.nseg * TILE_M * (p.TB + 1) * 4 + 15) / 16 * 16);
+    const size_t fixed = (size_t)p.yt_bytes + (2 * MAX_STAGES + 4) * 8 + 16 + (2 * TILE_M + 256 + 128) * 4;
+    int S = (int)((225 * 1024 - fixed) / stage);
+    if (S > MAX_STAGES) S = MAX_STAGES;
+    if (S < 2) return false;
+    p.nstages = S;
+    p.expanders = (TILE_M + p.n_mma + 31) / 32 * 32;
+    // one expander group and eight epilogue warps
+    p.groups = 1;
+    p.epi_warps = 8;
+    if (p.groups * p.expanders + 32 + 32 * p.epi_warps > MAX_THREADS) return false;
+    out->p = p;
+    out->smem = S * stage + fixed;
+    out->grid = dim3((unsigned)sms);
+    out->threads = p.groups * p.expanders + 32 + 32 * p.epi_warps;
+    out->persistent = true;
+    return out->smem <= 227 * 1024;
+}
 
 bool plan(const GemmArgs& a, TcPlan* out)
 {
@@ -498,7 +846,13 @@ bool plan(const GemmArgs& a, TcPlan* out)
     // two M tiles per CTA when their accumulators fit tensor memory and enough CTAs remain to fill the GPU
     const int mtiles = (p.units + p.UT - 1) / p.UT;
     const int btiles = (a.batch + p.TB - 1) / p.TB;
+    for (int sft = 0; sft < 8; ++sft) p.mul[sft] = 1u << (7 - sft);
+    p.mask_sign = 0x80808080u;
+    p.mask_half = 0x40404040u;
     p.MT = (2 * p.nseg * p.n_mma <= 512 && (long long)(mtiles / 2) * btiles >= 2 * 148) ? 2 : 1;
+    // with one M tile per CTA and more tiles than SMs, the persistent form hides the epilogues; with two M tiles
+    // per CTA the plain form's lower shared-memory traffic per MMA counts for more (measured)
+    if (p.MT == 1 && plan_persistent(p, mtiles, btiles, out)) return true;
     int cols = 32;
     while (cols < p.MT * p.nseg * p.n_mma) cols <<= 1;
     if (cols > 512) return false;
@@ -512,21 +866,20 @@ bool plan(const GemmArgs& a, TcPlan* out)
     p.nstages = S;
     p.expanders = (p.MT * TILE_M + p.n_mma + 31) / 32 * 32;
     p.groups = (2 * p.expanders + 32 <= MAX_THREADS) ? 2 : 1;
-    for (int sft = 0; sft < 8; ++sft) p.mul[sft] = 1u << (7 - sft);
-    p.mask_sign = 0x80808080u;
-    p.mask_half = 0x40404040u;
     out->p = p;
     out->smem = S * stage + (2 * MAX_STAGES + 1) * 8 + 24 + (2 * TILE_M + 256 + 128) * 4;   // stages, barriers, slot, coefficients
     out->grid = dim3((unsigned)((mtiles + p.MT - 1) / p.MT), (unsigned)btiles);
+    out->threads = p.groups * p.expanders + 32;
+    out->persistent = false;
     return out->grid.y <= 65535u && out->smem <= 227 * 1024;
 }
 
 template <int KA>
 amq_status launch_ka(const TcPlan& pl, cudaStream_t st)
 {
-    auto kernel = bgemm_tc_kernel<KA>;
+    auto kernel = pl.persistent ? bgemm_tc_persistent_kernel<KA> : bgemm_tc_kernel<KA>;
     AMQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
-    kernel<<<pl.grid, pl.p.groups * pl.p.expanders + 32, pl.smem, st>>>(pl.p);
+    kernel<<<pl.grid, pl.threads, pl.smem, st>>>(pl.p);
     AMQ_LAUNCH_CHECK();
     return AMQ_OK;
 }

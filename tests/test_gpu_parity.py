@@ -151,6 +151,9 @@ GEMM_CASES = [
     (40, 8192, 2, 2, 2),
     (2048, 2048, 2, 2, 5),               # few vectors, large matrix: one padded tile on the tensor cores
     (1031, 4096, 3, 2, 15),
+    (2500, 300, 4, 4, 70),               # more tiles than SMs, one M tile per CTA: the persistent tensor-core kernel
+    (2500, 100, 4, 4, 70),               # the same with a single pipeline step per tile
+    (6144, 200, 2, 3, 250),              # 384 tiles, ragged last batch tile
     # batch 1: the streaming matrix-vector kernel (segments of 1..32 lanes per row, one or two chunks per lane)
     (300, 8192, 3, 3, 1),
     (1000, 1024, 2, 3, 1),
@@ -217,6 +220,8 @@ CELL_CASES = [
     ("gru", 64, 40, 2, 3, 19),
     ("gru", 100, 129, 3, 2, 5),           # I not a multiple of 32: the column split falls inside a word
     ("gru", 33, 31, 1, 4, 2),
+    ("lstm", 40, 640, 4, 4, 70),          # 160 tiles: gate epilogues of the persistent tensor-core kernel
+    ("gru", 64, 800, 4, 1, 200),
     # batch 1 goes through the persistent weight-stationary kernel
     ("lstm", 1024, 1024, 2, 2, 1),        # the hidden-1024 layer of the benchmark, one step
     ("lstm", 1536, 1024, 3, 3, 1),        # n = 2560: sixteen elements per thread
