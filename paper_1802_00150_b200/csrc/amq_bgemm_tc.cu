@@ -214,7 +214,8 @@ __device__ __forceinline__ float logistic(float v) { return 1.0f / (1.0f + __exp
 // Epilogue, first half: tensor memory -> registers -> partial products y[plane-row][batch entry] in shared memory
 // (EPI_DOTS: the integer partials straight to global memory).  A thread is a plane-row (lane of tensor memory, lane
 // quarter `quarter` = warp index mod 4); the work items (M tile, column segment, 8 batch entries = 8 * KA columns)
-// are dealt out to `nslots` groups of four warps.  Reads of the accumulators are complete on return.
+// are dealt out to `nslots` groups of four warps (group s takes entries 8 s, 8 (s + nslots), .. of every M tile
+// and segment).  Reads of the accumulators are complete on return.
 template <int KA>
 __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_t tmem_acc, int u0, int b0, int quarter, int lane,
                                                       int slot, int nslots, const float* sAlpha, const float* sBeta,
@@ -225,14 +226,13 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
     const int TMp = p.UT * p.gates * k_w;
     const int pr = quarter * 32 + lane;
     const int groups = p.TB >> 3;
-    const int items1 = p.MT * p.nseg * groups;
     const uint32_t tlane = tmem_acc + ((uint32_t)(quarter * 32) << 16);
     if (a.epilogue == EPI_DOTS) {
         const int pad = p.wpr * 32 - a.n;
         const int l = pr / k_w, i = pr - l * k_w;
         const int gate = l % p.gates;
-        for (int item = slot; item < items1; item += nslots) {
-            const int g = item % groups, mt = item / groups;        // (one column segment in this epilogue)
+        for (int mt = 0; mt < p.MT; ++mt)                           // (one column segment in this epilogue)
+        for (int g = slot; g < groups; g += nslots) {
             const int u = u0 + mt * p.UT + l / p.gates;
             const bool row_ok = pr < TMp && u < p.units;
             const size_t row = (size_t)gate * p.units + u;
@@ -249,9 +249,11 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
         }
         return;
     }
-    for (int item = slot; item < items1; item += nslots) {
-        const int g = item % groups, ms = item / groups;            // ms = mt * nseg + seg
-        const int mt = ms / p.nseg, seg = ms - mt * p.nseg;
+    // loops without divisions: the per-item overhead is spread over only 8 * KA accumulators per thread
+    for (int mt = 0; mt < p.MT; ++mt)
+    for (int seg = 0; seg < p.nseg; ++seg)
+    for (int g = slot; g < groups; g += nslots) {
+        const int ms = mt * p.nseg + seg;
         int acc[KA][8];
 #pragma unroll
         for (int c = 0; c < KA; ++c) tmem_ld8(tlane + (uint32_t)(ms * n_mma + g * KA * 8 + c * 8), acc[c]);
@@ -309,13 +311,19 @@ __device__ __forceinline__ void epilogue_smem_to_global(const TcParams& p, const
             const float* y0 = Yt + ((size_t)(mt * p.nseg) * TILE_M + li * k_w) * ldy;
             const int bend = (a.batch - b0 < TB) ? a.batch - b0 : TB;
             int bb = bsub;
-            for (; bb + 3 * bstep < bend; bb += 4 * bstep) {       // four entries in flight
-                float s[4] = {bias, bias, bias, bias};
-                for (int i = 0; i < k_w; ++i)
+            float* out = a.y + (size_t)b0 * a.ldy + row;
+            for (; bb + 7 * bstep < bend; bb += 8 * bstep) {       // eight entries in flight, planes unrolled
+                float s[8];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) s[q] += y0[i * ldy + bb + q * bstep];
+                for (int q = 0; q < 8; ++q) {
+                    const float* yq = y0 + bb + q * bstep;
+                    s[q] = bias + yq[0];
+                    if (k_w > 1) s[q] += yq[ldy];
+                    if (k_w > 2) s[q] += yq[2 * ldy];
+                    if (k_w > 3) s[q] += yq[3 * ldy];
+                }
 #pragma unroll
-                for (int q = 0; q < 4; ++q) a.y[(size_t)(b0 + bb + q * bstep) * a.ldy + row] = s[q];
+                for (int q = 0; q < 8; ++q) out[(size_t)(bb + q * bstep) * a.ldy] = s[q];
             }
             for (; bb < bend; bb += bstep) {
                 float s = bias;
@@ -427,6 +435,9 @@ bgemm_tc_kernel(TcParams p)
         const int grp = tid / EXP, r_all = tid - grp * EXP;
         const uint4* src = nullptr;
         uint32_t dst0;                                              // shared address of the row in stage 0
+        const float* coef_src = nullptr;                            // the row's coefficient, staged for the epilogue
+        float* coef_dst = nullptr;
+        const float* corr_src = nullptr;                            // first of the KA coefficients of a batch entry
         if (r_all < MT * TILE_M) {
             const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
             size_t prow = 0;                                        // plane-row index in Wcodes / Walpha
@@ -439,8 +450,10 @@ bgemm_tc_kernel(TcParams p)
                 }
             }
             dst0 = smem_u32(stage_base) + r_all * 128;
-            // the row's coefficient, for the epilogue (its latency hides behind the main loop)
-            if (grp == 0) sAlpha[r_all] = (src && a.epilogue != EPI_DOTS) ? __ldg(a.Walpha + prow) : 0.0f;
+            if (grp == 0) {
+                coef_dst = sAlpha + r_all;
+                if (src && a.epilogue != EPI_DOTS) coef_src = a.Walpha + prow;
+            }
         } else {
             const int r = r_all - MT * TILE_M;
             const int b = b0 + r / KA, j = r % KA;
@@ -448,13 +461,9 @@ bgemm_tc_kernel(TcParams p)
             if (valid) src = reinterpret_cast<const uint4*>(a.xcodes + ((size_t)b * KA + j) * p.wpr);
             dst0 = smem_u32(stage_base) + a_stage_bytes + r * 128;
             if (grp == 0 && r < n_mma) {
-                const bool use = valid && a.epilogue != EPI_DOTS;
-                sBeta[r] = use ? __ldg(a.xbeta + (size_t)b * KA + j) : 0.0f;
-                if (j == 0) {
-                    float sum = 0.0f;
-                    for (int jj = 0; jj < KA; ++jj) sum += use ? __ldg(a.xbeta + (size_t)b * KA + jj) : 0.0f;
-                    sBcorr[r / KA] = -(float)(p.wpr * 32 - a.n) * sum;
-                }
+                coef_dst = sBeta + r;
+                if (valid && a.epilogue != EPI_DOTS) coef_src = a.xbeta + (size_t)b * KA + j;
+                if (j == 0) corr_src = coef_src;
             }
         }
         const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
@@ -469,6 +478,16 @@ bgemm_tc_kernel(TcParams p)
 
         uint4 cur = (src && grp < CH) ? __ldg(src + grp) : zero;    // own steps: grp, grp + G, ..
         uint4 nxt = (src && grp + G < CH) ? __ldg(src + grp + G) : zero;
+        // coefficients for the epilogue, after the first operand loads are under way (the stores below wait for
+        // their loads; the latency hides behind the main loop)
+        if (coef_dst) {
+            *coef_dst = coef_src ? __ldg(coef_src) : 0.0f;
+            if (r_all >= MT * TILE_M && (r_all - MT * TILE_M) % KA == 0) {
+                float sum = 0.0f;
+                for (int jj = 0; jj < KA; ++jj) sum += corr_src ? __ldg(corr_src + jj) : 0.0f;
+                sBcorr[(r_all - MT * TILE_M) / KA] = -(float)(p.wpr * 32 - a.n) * sum;
+            }
+        }
         int buf = grp;                                              // G <= S
         uint32_t empty_parity = 1;                                  // parity that means "never used" on the first lap
         for (int c = grp; c < CH; c += G) {
