@@ -258,6 +258,27 @@ AMQ_API amq_status amq_log_softmax_argmax(const float* logits, int rows, int n, 
                                   float* logp, int ldp, int32_t* argmax, void* stream);
 
 /*
+ * Greedy decoding with the language model of Eq. 6, one sequence, enqueued as one chain on `stream` (seven kernel
+ * launches per token, no host round trip).  For t = 0 .. steps-1:
+ *   x_t = row tokens[t] of the quantized embedding (We_codes [vocab][k_e][wpr(I)], We_alpha [vocab][k_e]);
+ *   (h, c) <- LSTM step in the paper's own form (W_i [4H x I], W_h [4H x H], k_w bits, bias [4H] or NULL; h quantized
+ *   on-line with k_a bits and T alternating rounds);
+ *   logits = W_s h_hat + bias_s (Ws_codes [vocab][k_s][wpr(H)], Ws_alpha [vocab][k_s], bias_s [vocab] or NULL);
+ *   logp[t][.] = log-softmax(logits) when logp is given; tokens[t + 1] = arg-max (first index among equal maxima).
+ * tokens: DEVICE int32 [steps + 1], tokens[0] set by the caller (ids outside [0, vocab) are clamped); h, c: DEVICE
+ * fp32 [H], start state in, state after the last step out; logp: DEVICE fp32 [steps][vocab] or NULL; workspace: DEVICE,
+ * amq_lm_decode_workspace_bytes(...) bytes, 16-byte aligned, owned by the caller, contents undefined between calls.
+ * Errors as for the calls it is made of; nothing is enqueued after the first failing launch.
+ */
+AMQ_API size_t amq_lm_decode_workspace_bytes(int vocab, int I, int H, int k_e, int k_a);
+AMQ_API amq_status amq_lm_greedy_decode(const uint32_t* We_codes, const float* We_alpha, int vocab, int I, int k_e,
+                                const uint32_t* Wi_codes, const float* Wi_alpha,
+                                const uint32_t* Wh_codes, const float* Wh_alpha, const float* bias, int H, int k_w,
+                                const uint32_t* Ws_codes, const float* Ws_alpha, const float* bias_s, int k_s,
+                                int k_a, int T, int32_t* tokens, int steps, float* h, float* c, float* logp,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The sequence calls with HOST activations and results: x_seq, h0, c0 are read from host memory
  * (pinned memory makes the copies asynchronous) into `staging`, the sequence runs, and h_last / c_last
  * (and h_seq when not NULL) are copied back to host memory; the call returns after the stream has

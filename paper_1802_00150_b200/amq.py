@@ -52,6 +52,9 @@ EXPORTS = {
     "amq_gru_sequence_host": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _int, _vp, _int, _int, _int,
                                      _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
     "amq_workspace_status": (_int, [_vp, _vp]),
+    "amq_lm_decode_workspace_bytes": (_sz, [_int, _int, _int, _int, _int]),
+    "amq_lm_greedy_decode": (_int, [_vp, _vp, _int, _int, _int, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp, _vp, _vp, _int,
+                                    _int, _int, _vp, _int, _vp, _vp, _vp, _vp, _sz, _vp]),
     "amq_log_softmax_argmax": (_int, [_vp, _int, _int, _int, _vp, _int, _vp, _vp]),
     "amq_embedding_rows": (_int, [_vp, _vp, _int, _int, _int, _vp, _int, _vp, _vp, _vp]),
     "amq_lstm_paper_workspace_bytes": (_sz, [_int, _int, _int, _int]),
@@ -337,11 +340,30 @@ def lstm_sequence_paper(Wi_codes, Wi_alpha, Wh_codes, Wh_alpha, bias, I, H, xcod
 
 
 def log_softmax_argmax(logits, want_logp=True, argmax=None):
-    """logits (rows, n) fp32 -> (log-probabilities (rows, n) or None, argmax (rows,) int32)."""
-    logits = _dev(logits, torch.float32, "logits")
+    """logits (rows, n) fp32, rows contiguous (any row stride) -> (log-probabilities (rows, n) or None, argmax (rows,) int32)."""
+    if not (isinstance(logits, torch.Tensor) and logits.is_cuda and logits.dtype == torch.float32 and logits.dim() == 2
+            and (logits.shape[1] == 1 or logits.stride(1) == 1)):
+        raise TypeError("logits must be a 2-D CUDA float32 tensor with contiguous rows")
     rows, n = logits.shape
-    logp = torch.empty_like(logits) if want_logp else None
+    ld = logits.stride(0) if rows > 1 else max(n, logits.stride(0))
+    logp = torch.empty((rows, n), dtype=torch.float32, device=logits.device) if want_logp else None
     argmax = torch.empty((rows,), dtype=torch.int32, device=logits.device) if argmax is None else argmax
-    _check(_lib.amq_log_softmax_argmax(_ptr(logits), rows, n, logits.stride(0) if rows > 1 else n, _ptr(logp), n,
-                                       _ptr(argmax), _stream()))
+    _check(_lib.amq_log_softmax_argmax(_ptr(logits), rows, n, ld, _ptr(logp), n, _ptr(argmax), _stream()))
     return logp, argmax
+
+
+def new_decode_workspace(vocab, I, H, k_e, k_a, device="cuda"):
+    return torch.empty((_lib.amq_lm_decode_workspace_bytes(vocab, I, H, k_e, k_a),), dtype=torch.uint8, device=device)
+
+
+def lm_greedy_decode(We_codes, We_alpha, Wi_codes, Wi_alpha, Wh_codes, Wh_alpha, bias, Ws_codes, Ws_alpha, bias_s, I, H,
+                     k_a, T, tokens, h, c, workspace, logp=None):
+    """tokens: int32 (steps + 1,), tokens[0] given, the rest written; h, c: (H,) or (1, H) fp32, updated in place."""
+    vocab, k_e = We_codes.shape[0], We_codes.shape[1]
+    k_w, k_s = Wi_codes.shape[1], Ws_codes.shape[1]
+    steps = tokens.numel() - 1
+    _check(_lib.amq_lm_greedy_decode(_ptr(We_codes), _ptr(We_alpha), vocab, I, k_e, _ptr(Wi_codes), _ptr(Wi_alpha),
+                                     _ptr(Wh_codes), _ptr(Wh_alpha), _ptr(bias), H, k_w, _ptr(Ws_codes), _ptr(Ws_alpha),
+                                     _ptr(bias_s), k_s, k_a, T, _ptr(tokens), steps, _ptr(h), _ptr(c), _ptr(logp),
+                                     _ptr(workspace), workspace.numel(), _stream()))
+    return tokens

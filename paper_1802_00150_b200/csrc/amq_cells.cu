@@ -39,18 +39,47 @@ amq_status enqueue_persistent(const CellCall& c, const CellWorkspace& ws, const 
                                  h0, c0, h_seq, h_last, c_last, ws.hx, ws.status, st);
 }
 
+__global__ void lstm_gates_kernel(const float* __restrict__ pre, const float* __restrict__ addend, const float* __restrict__ c_in,
+                                  float* __restrict__ h_out, float* __restrict__ c_out, int H)
+{
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= H) return;
+    float g4[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) g4[g] = pre[g * H + u] + (addend ? addend[g * H + u] : 0.0f);
+    const float ig = 1.0f / (1.0f + __expf(-g4[0])), fg = 1.0f / (1.0f + __expf(-g4[1])), og = 1.0f / (1.0f + __expf(-g4[2]));
+    const float c = fg * c_in[u] + ig * tanhf(g4[3]);
+    c_out[u] = c;
+    h_out[u] = og * tanhf(c);
+}
+
 // quantize z = [x ; h_in] into the workspace, then product + gates
 amq_status enqueue_step(const CellCall& c, const CellWorkspace& ws, const float* x, const float* h_in,
                         const float* c_in, float* h_out, float* c_out, cudaStream_t st)
 {
+    GemmArgs a{};
+    a.Wcodes = c.Wcodes; a.Walpha = c.Walpha; a.m = (c.gru ? 3 : 4) * c.H; a.n = c.I + c.H; a.k_w = c.k_w;
+    a.xcodes = ws.zcodes; a.xbeta = ws.zbeta; a.batch = c.batch; a.k_a = c.k_a;
+    a.bias = c.bias;
+    if (c.batch == 1 && !c.gru) {
+        // a single step of one LSTM sequence: quantizer, the bandwidth-bound matrix-vector kernel for the
+        // pre-activations (into the exchange buffer of the sequence kernel, 4H floats, unused here) and a small gate
+        // kernel: three plain launches cost less than the cooperative launch of the sequence kernel
+        a.epilogue = EPI_Y; a.y = reinterpret_cast<float*>(ws.hx); a.ldy = 4 * c.H;
+        if (gemv_supported(a)) {
+            amq_status s1 = launch_quantize(x, c.I, c.I, h_in, c.H, c.H, 1, c.k_a, c.T, ws.zcodes, ws.zbeta, st);
+            if (s1 != AMQ_OK) return s1;
+            s1 = launch_binary_gemv(a, st);
+            if (s1 != AMQ_OK) return s1;
+            return launch_lstm_gates(a.y, nullptr, c_in, h_out, c_out, c.H, st);
+        }
+        a.y = nullptr; a.ldy = 0;
+    }
     if (use_persistent(c))      // batch 1: one launch of the weight-stationary kernel, a sequence of one step
         return enqueue_persistent(c, ws, x, 1, h_in, c_in, nullptr, h_out, c_out, st);
     amq_status s = launch_quantize(x, c.I, c.I, h_in, c.H, c.H, c.batch, c.k_a, c.T, ws.zcodes, ws.zbeta, st);
     if (s != AMQ_OK) return s;
-    GemmArgs a{};
-    a.Wcodes = c.Wcodes; a.Walpha = c.Walpha; a.m = (c.gru ? 3 : 4) * c.H; a.n = c.I + c.H; a.k_w = c.k_w;
-    a.xcodes = ws.zcodes; a.xbeta = ws.zbeta; a.batch = c.batch; a.k_a = c.k_a;
-    a.bias = c.bias; a.epilogue = c.gru ? EPI_GRU : EPI_LSTM;
+    a.epilogue = c.gru ? EPI_GRU : EPI_LSTM;
     a.I = c.I; a.H = c.H; a.h_in = h_in; a.c_in = c_in; a.h_out = h_out; a.c_out = c_out;
     return launch_binary_gemm(a, st);
 }
@@ -144,6 +173,15 @@ amq_status sequence_host_entry(const CellCall& c, const float* x_seq_host, int s
 }
 
 }  // namespace
+
+amq_status launch_lstm_gates(const float* pre, const float* addend, const float* c_in, float* h_out, float* c_out, int H,
+                             cudaStream_t st)
+{
+    lstm_gates_kernel<<<(unsigned)((H + 255) / 256), 256, 0, st>>>(pre, addend, c_in, h_out, c_out, H);
+    AMQ_LAUNCH_CHECK();
+    return AMQ_OK;
+}
+
 }  // namespace amq
 
 extern "C" {

@@ -19,6 +19,7 @@ struct PaperWorkspace {
     float* proj;        // [steps][batch][4H]  W_i x_t + bias
     float* h[2];        // [batch][H] ping / pong
     float* c;           // [batch][H]
+    float* gates;       // [4H] pre-activations of a single sequence (batch 1)
     size_t bytes;
 };
 
@@ -33,6 +34,7 @@ PaperWorkspace carve(void* base, int H, int batch, int steps, int k_a)
     w.h[0] = reinterpret_cast<float*>(p + off);      off += round_up((size_t)batch * H * 4, 256);
     w.h[1] = reinterpret_cast<float*>(p + off);      off += round_up((size_t)batch * H * 4, 256);
     w.c = reinterpret_cast<float*>(p + off);         off += round_up((size_t)batch * H * 4, 256);
+    w.gates = reinterpret_cast<float*>(p + off);     off += round_up((size_t)4 * H * 4, 256);
     w.bytes = off;
     return w;
 }
@@ -74,7 +76,18 @@ amq_status recurrent_part(const PaperCall& c, const PaperWorkspace& ws, const fl
     GemmArgs a{};
     a.Wcodes = c.Wh_codes; a.Walpha = c.Wh_alpha; a.m = 4 * c.H; a.n = c.H; a.k_w = c.k_w;
     a.xcodes = ws.hcodes; a.xbeta = ws.hbeta; a.batch = c.batch; a.k_a = c.k_a;
-    a.bias = nullptr; a.epilogue = EPI_LSTM;
+    a.bias = nullptr;
+    if (c.batch == 1) {
+        // one sequence: the bandwidth-bound matrix-vector kernel writes the pre-activations, a small kernel applies the gates
+        a.epilogue = EPI_Y; a.y = ws.gates; a.ldy = 4 * c.H;
+        if (gemv_supported(a)) {
+            s = launch_binary_gemv(a, st);
+            if (s != AMQ_OK) return s;
+            return launch_lstm_gates(ws.gates, proj, c_in, h_out, c_out, c.H, st);
+        }
+    }
+    a.y = nullptr; a.ldy = 0;
+    a.epilogue = EPI_LSTM;
     a.I = 0; a.H = c.H; a.h_in = h_in; a.c_in = c_in; a.h_out = h_out; a.c_out = c_out;
     a.addend = proj; a.ld_addend = 4 * c.H;
     return launch_binary_gemm(a, st);

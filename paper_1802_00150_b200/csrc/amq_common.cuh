@@ -92,6 +92,9 @@ struct GemmArgs {
 amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st);
 
 // Batch-1 streaming kernel (EPI_DOTS / EPI_Y): whether it covers a problem, and its launch.
+// gates of Eq. 6 for one sequence from pre-activations pre[4H] (+ addend[4H] when given), rows i, f, o, g
+amq_status launch_lstm_gates(const float* pre, const float* addend, const float* c_in, float* h_out, float* c_out, int H,
+                             cudaStream_t st);
 bool gemv_supported(const GemmArgs& a);
 amq_status launch_binary_gemv(const GemmArgs& a, cudaStream_t st);
 

@@ -1,0 +1,90 @@
+// Greedy decoding with the quantized language model of Eq. 6 (one sequence, the arg-max token fed back), enqueued
+// as one chain on the caller's stream: per token the embedding row (pre-quantized, needs no further quantization),
+// the input projection W_i x + b, the recurrent product W_h h_hat on the on-line quantized state, the gates, the
+// quantizer on the new state (its planes serve the output layer now and the recurrence of the next token), the
+// output product W_s h_hat + b_s and log-softmax / arg-max.  Seven launches per token, no host round trip.
+#include "amq_common.cuh"
+
+namespace amq {
+namespace {
+
+struct DecodeWorkspace {
+    uint32_t* xcodes;   // [k_e][wpr(I)]
+    float* xbeta;       // [k_e]
+    uint32_t* hcodes;   // [k_a][wpr(H)]
+    float* hbeta;       // [k_a]
+    float* proj;        // [4H]
+    float* pre;         // [4H]
+    float* logits;      // [vocab]
+    size_t bytes;
+};
+
+DecodeWorkspace carve(void* base, int vocab, int I, int H, int k_e, int k_a)
+{
+    DecodeWorkspace w;
+    char* p = static_cast<char*>(base);
+    size_t off = 0;
+    w.xcodes = reinterpret_cast<uint32_t*>(p + off); off += round_up((size_t)k_e * words_per_row(I) * 4, 256);
+    w.xbeta = reinterpret_cast<float*>(p + off);     off += 256;
+    w.hcodes = reinterpret_cast<uint32_t*>(p + off); off += round_up((size_t)k_a * words_per_row(H) * 4, 256);
+    w.hbeta = reinterpret_cast<float*>(p + off);     off += 256;
+    w.proj = reinterpret_cast<float*>(p + off);      off += round_up((size_t)4 * H * 4, 256);
+    w.pre = reinterpret_cast<float*>(p + off);       off += round_up((size_t)4 * H * 4, 256);
+    w.logits = reinterpret_cast<float*>(p + off);    off += round_up((size_t)vocab * 4, 256);
+    w.bytes = off;
+    return w;
+}
+
+}  // namespace
+}  // namespace amq
+
+extern "C" {
+
+size_t amq_lm_decode_workspace_bytes(int vocab, int I, int H, int k_e, int k_a)
+{
+    if (vocab < 1 || I < 1 || H < 1 || !amq::valid_k(k_e) || !amq::valid_k(k_a)) return 0;
+    return amq::carve(nullptr, vocab, I, H, k_e, k_a).bytes;
+}
+
+amq_status amq_lm_greedy_decode(const uint32_t* We_codes, const float* We_alpha, int vocab, int I, int k_e,
+                                const uint32_t* Wi_codes, const float* Wi_alpha, const uint32_t* Wh_codes, const float* Wh_alpha,
+                                const float* bias, int H, int k_w,
+                                const uint32_t* Ws_codes, const float* Ws_alpha, const float* bias_s, int k_s,
+                                int k_a, int T, int32_t* tokens, int steps, float* h, float* c, float* logp,
+                                void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!We_codes || !We_alpha || !Wi_codes || !Wi_alpha || !Wh_codes || !Wh_alpha || !Ws_codes || !Ws_alpha || vocab < 1 ||
+        I < 1 || H < 1 || steps < 0)
+        return AMQ_ERR_INVALID_ARG;
+    if (!amq::valid_k(k_e) || !amq::valid_k(k_w) || !amq::valid_k(k_s) || !amq::valid_k(k_a) || T < 0 || I > AMQ_MAX_N ||
+        H > AMQ_MAX_N)
+        return AMQ_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < amq_lm_decode_workspace_bytes(vocab, I, H, k_e, k_a)) return AMQ_ERR_WORKSPACE;
+    if (!amq::aligned16(workspace) || !amq::aligned16(We_codes) || !amq::aligned16(Wi_codes) || !amq::aligned16(Wh_codes) ||
+        !amq::aligned16(Ws_codes))
+        return AMQ_ERR_ALIGNMENT;
+    if (steps == 0) return AMQ_OK;
+    if (!tokens || !h || !c) return AMQ_ERR_INVALID_ARG;
+    const amq::DecodeWorkspace ws = amq::carve(workspace, vocab, I, H, k_e, k_a);
+    cudaStream_t st = (cudaStream_t)stream;
+    amq_status s = amq_quantize(h, 1, H, H, k_a, T, ws.hcodes, ws.hbeta, stream);          // h_hat of the start state
+    for (int t = 0; t < steps && s == AMQ_OK; ++t) {
+        s = amq_embedding_rows(We_codes, We_alpha, vocab, I, k_e, tokens + t, 1, ws.xcodes, ws.xbeta, stream);
+        if (s != AMQ_OK) break;
+        s = amq_binary_gemm(Wi_codes, Wi_alpha, 4 * H, I, k_w, ws.xcodes, ws.xbeta, 1, k_e, bias, ws.proj, 4 * H, stream);
+        if (s != AMQ_OK) break;
+        s = amq_binary_gemm(Wh_codes, Wh_alpha, 4 * H, H, k_w, ws.hcodes, ws.hbeta, 1, k_a, nullptr, ws.pre, 4 * H, stream);
+        if (s != AMQ_OK) break;
+        s = amq::launch_lstm_gates(ws.pre, ws.proj, c, h, c, H, st);                        // state updated in place
+        if (s != AMQ_OK) break;
+        s = amq_quantize(h, 1, H, H, k_a, T, ws.hcodes, ws.hbeta, stream);
+        if (s != AMQ_OK) break;
+        s = amq_binary_gemm(Ws_codes, Ws_alpha, vocab, H, k_s, ws.hcodes, ws.hbeta, 1, k_a, bias_s, ws.logits, vocab, stream);
+        if (s != AMQ_OK) break;
+        s = amq_log_softmax_argmax(ws.logits, 1, vocab, vocab, logp ? logp + (size_t)t * vocab : nullptr, vocab, tokens + t + 1,
+                                   stream);
+    }
+    return s;
+}
+
+}  // extern "C"

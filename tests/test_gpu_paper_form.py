@@ -83,12 +83,18 @@ def test_paper_form_sequence_and_steps(amq, I, H, kw, ke, ka, batch, steps):
     assert drift <= 0.05
 
 
-@pytest.mark.parametrize("rows,n", [(1, 42000), (7, 1000), (3, 33), (2, 1)])
-def test_log_softmax_argmax(amq, rows, n):
+@pytest.mark.parametrize("rows,n,ld", [(1, 42000, 42000), (7, 1000, 1000), (3, 33, 33), (2, 1, 1), (3, 1001, 1004),
+                                       (2, 4099, 4100), (2, 50001, 50004), (2, 49152, 49152)])
+def test_log_softmax_argmax(amq, rows, n, ld):
+    """Rows read once into registers (aligned rows up to 49152 logits, with and without a ragged tail) and the
+    three-pass kernel (longer or unaligned rows)."""
     z = synth.normal((rows, n), 3.0, 95 + n, 1)
     if n > 400:
         z[0, 17] = z[0, 400] = z[0].max() + 1.0                 # equal maxima: the first index wins
-    logp, arg = amq.log_softmax_argmax(dev(z))
+        z[-1, n - 1] = z[-1].max() + 2.0                        # the maximum in the ragged tail
+    wide = torch.full((rows, ld), float("nan"), device="cuda")
+    wide[:, :n] = dev(z)
+    logp, arg = amq.log_softmax_argmax(wide[:, :n])
     ref, rarg = oracle.log_softmax_argmax(z.astype(np.float64))
     assert np.abs(logp.cpu().numpy() - ref).max() <= 2e-5       # fp32 sum of up to 42000 exponentials + one log
     assert np.array_equal(arg.cpu().numpy(), rarg)
@@ -133,3 +139,48 @@ def test_output_layer_at_vocabulary_scale_and_greedy_decoding(amq):
             assert z_o[0, tok_g] >= top2[1] - 2 * tol           # otherwise any near-maximal token is valid
         tok_o = tok_g                                           # follow the library's choice
         ho, co = h.cpu().numpy().astype(np.float64), c.cpu().numpy().astype(np.float64)
+
+
+def test_native_greedy_decoding_equals_the_composed_calls_and_the_oracle_on_its_first_step(amq):
+    """amq_lm_greedy_decode enqueues the same kernels as the call-by-call loop above (checked there against the oracle
+    at every step): tokens, states and log-probabilities must agree bit for bit; the first step is also held against
+    the oracle directly."""
+    I, H, V, kw, ke, ka, steps = 96, 160, 3001, 3, 2, 2, 6
+    (Wic, Wia), (Whc, Wha), _, bias = model(I, H, 8, kw, ke, 131)
+    Wsc, Wsa = oracle.quantize_rows(synth.normal((V, H), 0.08, 131, 7).astype(np.float64), kw, 2)
+    Wec, Wea = oracle.quantize_rows(synth.normal((V, I), 0.5, 131, 8).astype(np.float64), ke, 2)
+    bs = synth.normal((V,), 0.1, 131, 9)
+    h0 = synth.uniform((1, H), -1, 1, 131, 10)
+    c0 = synth.uniform((1, H), -1, 1, 131, 11)
+    d = dict(Wic=cdev(Wic), Wia=dev(Wia), Whc=cdev(Whc), Wha=dev(Wha), bias=dev(bias), Wsc=cdev(Wsc), Wsa=dev(Wsa),
+             bs=dev(bs), Wec=cdev(Wec), Wea=dev(Wea))
+    # native loop
+    tokens = torch.zeros((steps + 1,), dtype=torch.int32, device="cuda")
+    tokens[0] = 77
+    h, c = dev(h0), dev(c0)
+    logp = torch.empty((steps, V), device="cuda")
+    ws = amq.new_decode_workspace(V, I, H, ke, ka)
+    amq.lm_greedy_decode(d["Wec"], d["Wea"], d["Wic"], d["Wia"], d["Whc"], d["Wha"], d["bias"], d["Wsc"], d["Wsa"], d["bs"],
+                         I, H, ka, 2, tokens, h, c, ws, logp=logp)
+    assert amq.device_status() == 0
+    # the same steps call by call
+    pws = amq.new_paper_workspace(H, 1, 1, ka)
+    tok = torch.tensor([77], dtype=torch.int32, device="cuda")
+    h2, c2 = dev(h0), dev(c0)
+    for t in range(steps):
+        xc, xb = amq.embedding_rows(d["Wec"], d["Wea"], I, tok)
+        h2, c2 = amq.lstm_step_paper(d["Wic"], d["Wia"], d["Whc"], d["Wha"], d["bias"], I, H, xc, xb, h2, c2, ka, 2, pws)
+        hc, hb = amq.quantize(h2, ka, 2)
+        logits = amq.binary_gemm(d["Wsc"], d["Wsa"], hc, hb, H, bias=d["bs"])
+        lp, tok = amq.log_softmax_argmax(logits)
+        assert int(tok[0]) == int(tokens[t + 1]), t
+        assert torch.equal(lp[0], logp[t]), t
+    assert torch.equal(h2, h) and torch.equal(c2, c)
+    # first step against the oracle
+    ho, co = oracle.lstm_step_paper(Wic, Wia, Whc, Wha, bias, I, H, Wec[[77]], Wea[[77]], h0.astype(np.float64),
+                                    c0.astype(np.float64), ka, 2)
+    hc_o, hb_o = oracle.quantize_rows(ho, ka, 2)
+    z_o = oracle.binary_gemm(Wsc, Wsa, hc_o, hb_o, H, bs.astype(np.float64))
+    lp_o, _ = oracle.log_softmax_argmax(z_o)
+    tol = parity.output_tolerance(Wsa, hb_o, H).max()
+    assert np.abs(logp[0].cpu().numpy() - lp_o[0]).max() <= 2 * tol + 2e-5
