@@ -514,6 +514,7 @@ def batched_lines(amq, torch, dev, flush, hbm_peak, peak_kind):
         del W, Wcodes, Walpha, acts, xc, xb, y
     out.append(paper_form_line(amq, torch, dev))
     out.append(greedy_decoding_line(amq, torch, dev))
+    out.extend(table6_lines(amq, torch, dev, flush))
     return out
 
 
@@ -544,6 +545,37 @@ def paper_form_line(amq, torch, dev):
                         "one batched input projection + per-step quantize(h) and W_h product)" % (batch, steps),
             "ms": ms, "bound": "tensor+latency", "us_per_timestep": 1e3 * ms / steps,
             "timesteps_per_s": batch * steps / (ms * 1e-3)}
+
+
+def table6_lines(amq, torch, dev, flush):
+    """The two matrix-vector shapes the paper times on one CPU core (Table 6): on-line quantization of the
+    1024-vector h plus the binary product, 4096 x 1024 (W_h h) and 42000 x 1024 (W_s h), at 2/2 and 3/3 bits.
+    Cold = L2 flushed before every run; warm = back to back.  The paper's CPU times are quoted for context only."""
+    paper_ms = {(4096, 2): 0.35, (4096, 3): 0.72, (42000, 2): 3.17, (42000, 3): 6.46}
+    out = []
+    for m in (4096, 42000):
+        for k in (2, 3):
+            n = 1024
+            g = torch.Generator(device=dev)
+            g.manual_seed(4)
+            Wc, Wa = amq.quantize(torch.randn((m, n), device=dev, generator=g) * 0.05, k, 2)
+            hvec = torch.rand((1, n), device=dev, generator=g) * 2 - 1
+            hc, hb = amq.quantize(hvec, k, 2)
+            y = torch.empty((1, m), device=dev)
+
+            def run():
+                amq.quantize(hvec, k, 2, codes=hc, coeffs=hb)
+                amq.binary_gemm(Wc, Wa, hc, hb, n, y=y)
+
+            for _ in range(3):
+                run()
+            cold = _event_ms(torch, run, flush, 10)
+            warm = _burst_ms(torch, run, 50)
+            out.append({"workload": "Table 6 shape: quantize(h) + binary product %d x %d, %d/%d bits, batch 1" % (m, n, k, k),
+                        "ms_cold": cold, "ms_warm": warm, "bound": "latency (two launches)",
+                        "paper_cpu_ms_one_xeon_core": paper_ms[(m, k)]})
+            del Wc, Wa
+    return out
 
 
 def greedy_decoding_line(amq, torch, dev):

@@ -61,20 +61,6 @@ amq_status enqueue_step(const CellCall& c, const CellWorkspace& ws, const float*
     a.Wcodes = c.Wcodes; a.Walpha = c.Walpha; a.m = (c.gru ? 3 : 4) * c.H; a.n = c.I + c.H; a.k_w = c.k_w;
     a.xcodes = ws.zcodes; a.xbeta = ws.zbeta; a.batch = c.batch; a.k_a = c.k_a;
     a.bias = c.bias;
-    if (c.batch == 1 && !c.gru) {
-        // a single step of one LSTM sequence: quantizer, the bandwidth-bound matrix-vector kernel for the
-        // pre-activations (into the exchange buffer of the sequence kernel, 4H floats, unused here) and a small gate
-        // kernel: three plain launches cost less than the cooperative launch of the sequence kernel
-        a.epilogue = EPI_Y; a.y = reinterpret_cast<float*>(ws.hx); a.ldy = 4 * c.H;
-        if (gemv_supported(a)) {
-            amq_status s1 = launch_quantize(x, c.I, c.I, h_in, c.H, c.H, 1, c.k_a, c.T, ws.zcodes, ws.zbeta, st);
-            if (s1 != AMQ_OK) return s1;
-            s1 = launch_binary_gemv(a, st);
-            if (s1 != AMQ_OK) return s1;
-            return launch_lstm_gates(a.y, nullptr, c_in, h_out, c_out, c.H, st);
-        }
-        a.y = nullptr; a.ldy = 0;
-    }
     if (use_persistent(c))      // batch 1: one launch of the weight-stationary kernel, a sequence of one step
         return enqueue_persistent(c, ws, x, 1, h_in, c_in, nullptr, h_out, c_out, st);
     amq_status s = launch_quantize(x, c.I, c.I, h_in, c.H, c.H, c.batch, c.k_a, c.T, ws.zcodes, ws.zbeta, st);
