@@ -37,6 +37,8 @@ _bst = _sig("amq_oracle_bst", None, _dp, _int, _int, _dp, _i8p)
 _obj = _sig("amq_oracle_objective", ctypes.c_double, _dp, _int, _int, _dp, _i8p)
 _quant = _sig("amq_oracle_quantize", None, _dp, _int, _int, _int, _dp, _i8p, _dp)
 _refined = _sig("amq_oracle_refined_greedy", None, _dp, _int, _int, _dp, _i8p)
+_qvar = _sig("amq_oracle_quantize_variant", None, _dp, _int, _int, _int, _int, _int, _dp, _i8p)
+_qrows_var = _sig("amq_oracle_quantize_rows_variant", None, _dp, _int, _int, _int, _int, _int, _int, _int, _u32p, _dp)
 _wpr = _sig("amq_oracle_words_per_row", _int, _int)
 _pack = _sig("amq_oracle_pack_plane", None, _i8p, _int, _u32p)
 _unpack = _sig("amq_oracle_unpack_plane", None, _u32p, _int, _i8p)
@@ -134,6 +136,28 @@ def refined_greedy(w, k):
     b = np.zeros((k, n), dtype=np.int8)
     _refined(_p(w, _dp), n, k, _p(alpha, _dp), _p(b, _i8p))
     return alpha, b
+
+
+METHOD_ALTERNATING, METHOD_REFINED_GREEDY = 0, 1
+
+
+def quantize_variant(w, k, T, method=METHOD_ALTERNATING, final_refit=False):
+    w = _d(w).ravel()
+    n = w.size
+    alpha = np.zeros(k)
+    b = np.zeros((k, n), dtype=np.int8)
+    _qvar(_p(w, _dp), n, k, T, method, int(final_refit), _p(alpha, _dp), _p(b, _i8p))
+    return alpha, b
+
+
+def quantize_rows_variant(x, k, T, method=METHOD_ALTERNATING, final_refit=False):
+    """x (rows, n) -> codes (rows, k, wpr) uint32, coeffs (rows, k) float64."""
+    x = _d(x)
+    rows, n = x.shape
+    codes = np.zeros((rows, k, words_per_row(n)), dtype=np.uint32)
+    coeffs = np.zeros((rows, k))
+    _qrows_var(_p(x, _dp), rows, n, n, k, T, method, int(final_refit), _p(codes, _u32p), _p(coeffs, _dp))
+    return codes, coeffs
 
 
 def pack_plane(b):

@@ -198,6 +198,36 @@ void amq_oracle_refined_greedy(const double* w, int n, int k, double* alpha, int
     free(r);
 }
 
+/* Variants of the quantizer (Sec. 2-3), for the comparison of Tables 1-2 and for the other reading of the
+ * order of the two half steps:
+ *   method 0: Algorithm 2 (greedy start, T alternating cycles); method 1: refined greedy (T ignored);
+ *   final_refit != 0: one more coefficient refit (Eq. 5) on the final codes, so that the returned alpha is
+ *   optimal for the returned b (Algorithm 2 as printed ends on the code update instead). */
+void amq_oracle_quantize_variant(const double* w, int n, int k, int T, int method, int final_refit,
+                                 double* alpha, int8_t* b)
+{
+    if (method == 1) amq_oracle_refined_greedy(w, n, k, alpha, b);
+    else amq_oracle_quantize(w, n, k, T, alpha, b, NULL);
+    if (final_refit) amq_oracle_ls_refit(w, n, k, b, alpha);
+}
+
+void amq_oracle_quantize_rows_variant(const double* x, int rows, int n, int ldx, int k, int T, int method,
+                                      int final_refit, uint32_t* codes, double* coeffs)
+{
+    int wpr = 4 * ((n + 127) / 128);
+    int8_t* b = (int8_t*)malloc((size_t)k * (size_t)(n > 0 ? n : 1));
+    for (int r = 0; r < rows; ++r) {
+        amq_oracle_quantize_variant(x + (size_t)r * ldx, n, k, T, method, final_refit, coeffs + (size_t)r * k, b);
+        for (int i = 0; i < k; ++i) {
+            uint32_t* words = codes + ((size_t)r * k + i) * wpr;
+            for (int q = 0; q < wpr; ++q) words[q] = 0u;
+            for (int t = 0; t < n; ++t)
+                if (b[(size_t)i * n + t] > 0) words[t >> 5] |= 1u << (t & 31);
+        }
+    }
+    free(b);
+}
+
 /* ---------------------------------------------------------------------------------------------
  * Bit packing of one +-1 plane (storage for the XNOR / bitcount product of Appendix A).
  * ------------------------------------------------------------------------------------------- */

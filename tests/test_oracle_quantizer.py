@@ -328,3 +328,35 @@ def test_cost_model_matches_the_paper(golden_dir):
     # quantizer: 2Tk^2 n binary + 2(T+1)kn non-binary; at T=2 the product model's 4k^2 n and 6kn terms
     b, nb = oracle.quantizer_ops(1024, 3, 2)
     assert b == 4 * 9 * 1024 and nb == 6 * 3 * 1024
+
+
+def test_variants_final_refit_and_refined_greedy():
+    """The variants of the comparison (Sec. 2, Tables 1-2) and the other reading of the order of the half steps.
+    Final refit: the codes are those of Algorithm 2, the coefficients solve the normal equations for those codes
+    (checked with numpy's least squares, an independent routine), and the error does not grow.  Refined greedy:
+    equals greedy bits re-solved after every bit, i.e. its coefficients solve the normal equations of its own codes."""
+    rng = np.random.default_rng(5)
+    for k in (1, 2, 3, 4):
+        for dist in ("normal", "heavy"):
+            w = rng.standard_normal(257) if dist == "normal" else rng.standard_normal(257) ** 3
+            a0, b0 = oracle.quantize(w, k, 2)
+            a1, b1 = oracle.quantize_variant(w, k, 2, oracle.METHOD_ALTERNATING, True)
+            assert np.array_equal(b0, b1)
+            lsq = np.linalg.lstsq(b1.T.astype(np.float64), w, rcond=None)[0]
+            if np.linalg.matrix_rank(b1.T.astype(np.float64)) == k:
+                assert np.allclose(a1, lsq, rtol=1e-9, atol=1e-12)
+            assert oracle.objective(w, a1, b1) <= oracle.objective(w, a0, b0) * (1 + 1e-12)
+            a2, b2 = oracle.quantize_variant(w, k, 7, oracle.METHOD_REFINED_GREEDY, False)      # T is ignored
+            ar, br = oracle.refined_greedy(w, k)
+            assert np.array_equal(b2, br) and np.array_equal(a2, ar)
+            if np.linalg.matrix_rank(br.T.astype(np.float64)) == k:
+                assert np.allclose(ar, np.linalg.lstsq(br.T.astype(np.float64), w, rcond=None)[0], rtol=1e-9, atol=1e-12)
+            # first bit of the refined method is the plain 1-bit fit
+            assert np.array_equal(br[0], np.where(w >= 0, 1, -1))
+    # rows form: the same through the packed layout
+    x = rng.standard_normal((5, 131))
+    codes, coeffs = oracle.quantize_rows_variant(x, 3, 2, oracle.METHOD_ALTERNATING, True)
+    for r in range(5):
+        a, b = oracle.quantize_variant(x[r], 3, 2, oracle.METHOD_ALTERNATING, True)
+        assert np.array_equal(coeffs[r], a)
+        assert np.array_equal(codes[r], oracle.pack_planes(b))
