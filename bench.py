@@ -515,6 +515,7 @@ def batched_lines(amq, torch, dev, flush, hbm_peak, peak_kind):
     out.append(paper_form_line(amq, torch, dev))
     out.append(greedy_decoding_line(amq, torch, dev))
     out.extend(table6_lines(amq, torch, dev, flush))
+    out.append(quality_line(amq, torch, dev))
     return out
 
 
@@ -575,6 +576,32 @@ def table6_lines(amq, torch, dev, flush):
                         "ms_cold": cold, "ms_warm": warm, "bound": "latency (two launches)",
                         "paper_cpu_ms_one_xeon_core": paper_ms[(m, k)]})
             del Wc, Wa
+    return out
+
+
+def quality_line(amq, torch, dev):
+    """Relative mean squared error ||w - w_hat||^2 / ||w||^2 of the quantization methods compared in Sec. 2 / Tables 1-2
+    (greedy, refined greedy, alternating with T = 2, and alternating followed by a last coefficient refit), on
+    synthetic rows (256 x 1024): Gaussian, and heavy-tailed (cube of a Gaussian).  A quality report, not a timing."""
+    g = torch.Generator(device=dev)
+    g.manual_seed(5)
+    base = torch.randn((256, 1024), device=dev, generator=g)
+    out = {"workload": "relative MSE of the quantization methods, 256 rows x 1024, computed with the library",
+           "bound": "none (quality report)"}
+    for name, w in (("gaussian", base * 0.03), ("heavy_tailed", base ** 3)):
+        norm = (w.double() ** 2).sum()
+        table = {}
+        for k in (2, 3, 4):
+            row = {}
+            for label, T, method, final in (("greedy", 0, amq.METHOD_ALTERNATING, False),
+                                            ("refined_greedy", 0, amq.METHOD_REFINED_GREEDY, False),
+                                            ("alternating_T2", 2, amq.METHOD_ALTERNATING, False),
+                                            ("alternating_T2_final_refit", 2, amq.METHOD_ALTERNATING, True)):
+                codes, coeffs = amq.quantize_variant(w, k, T, method, final)
+                w_hat = amq.unpack(codes, coeffs, 1024)
+                row[label] = float(((w.double() - w_hat.double()) ** 2).sum() / norm)
+            table["k=%d" % k] = row
+        out[name] = table
     return out
 
 

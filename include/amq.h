@@ -88,6 +88,20 @@ AMQ_API amq_status amq_quantize(const float* x, int rows, int n, int ldx, int k,
                         uint32_t* codes, float* coeffs, void* stream);
 
 /*
+ * Variants of the row quantizer (the comparison of Sec. 2 and Tables 1-2; the other reading of the order of
+ * Algorithm 2's half steps).  Arguments, layouts and errors as amq_quantize, plus
+ *   method:      AMQ_METHOD_ALTERNATING (Algorithm 2: greedy start, T cycles) or AMQ_METHOD_REFINED_GREEDY (after every
+ *                greedy bit all coefficients so far are re-solved by Eq. 5; T is ignored); anything else: AMQ_ERR_UNSUPPORTED;
+ *   final_refit: nonzero = one more coefficient refit (Eq. 5) on the final codes (Algorithm 2 as printed ends on the
+ *                code update, so its coefficients are those of the refit BEFORE the last code update).
+ * (AMQ_METHOD_ALTERNATING, 0) is amq_quantize itself; the other combinations run a general, slower kernel.
+ */
+#define AMQ_METHOD_ALTERNATING 0
+#define AMQ_METHOD_REFINED_GREEDY 1
+AMQ_API amq_status amq_quantize_variant(const float* x, int rows, int n, int ldx, int k, int T, int method, int final_refit,
+                                uint32_t* codes, float* coeffs, void* stream);
+
+/*
  * Pack sign planes given as floats into the bit layout above (storage for the XNOR / bit-count
  * product, Appendix A).  planes [rows][k][n] fp32, value >= 0 -> bit 1.  codes [rows][k][wpr] out.
  */

@@ -52,6 +52,7 @@ EXPORTS = {
     "amq_gru_sequence_host": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _int, _vp, _int, _int, _int,
                                      _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
     "amq_workspace_status": (_int, [_vp, _vp]),
+    "amq_quantize_variant": (_int, [_vp, _int, _int, _int, _int, _int, _int, _int, _vp, _vp, _vp]),
     "amq_lm_decode_workspace_bytes": (_sz, [_int, _int, _int, _int, _int]),
     "amq_lm_greedy_decode": (_int, [_vp, _vp, _int, _int, _int, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp, _vp, _vp, _int,
                                     _int, _int, _vp, _int, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -367,3 +368,19 @@ def lm_greedy_decode(We_codes, We_alpha, Wi_codes, Wi_alpha, Wh_codes, Wh_alpha,
                                      _ptr(bias_s), k_s, k_a, T, _ptr(tokens), steps, _ptr(h), _ptr(c), _ptr(logp),
                                      _ptr(workspace), workspace.numel(), _stream()))
     return tokens
+
+
+METHOD_ALTERNATING, METHOD_REFINED_GREEDY = 0, 1
+
+
+def quantize_variant(x, k, T, method=METHOD_ALTERNATING, final_refit=False):
+    """As quantize, with the method (alternating / refined greedy) and an optional last coefficient refit."""
+    if not (x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.stride(1) == 1):
+        raise TypeError("x must be a 2-D CUDA fp32 tensor with unit column stride")
+    rows, n = x.shape
+    ldx = x.stride(0) if rows > 1 else max(n, x.stride(0))
+    codes = _new_codes(rows, k, n, x.device)
+    coeffs = torch.empty((rows, k), dtype=torch.float32, device=x.device)
+    _check(_lib.amq_quantize_variant(_ptr(x), rows, n, ldx, k, T, method, int(final_refit), _ptr(codes), _ptr(coeffs),
+                                     _stream()))
+    return codes, coeffs

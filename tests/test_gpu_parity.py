@@ -347,3 +347,48 @@ def test_empty_batch_and_zero_steps(amq):
     assert torch.equal(h_last, h0) and torch.equal(c_last, c0)
     codes, coeffs = amq.quantize(torch.empty((0, 64), device="cuda"), 2, 2)
     assert codes.shape[0] == 0
+
+
+@pytest.mark.parametrize("method,final_refit", [(0, True), (1, False), (1, True)])
+@pytest.mark.parametrize("rows,n,k,dist", [(40, 600, 2, "normal"), (33, 1024, 3, "heavy"), (9, 4100, 4, "normal"),
+                                           (21, 131, 1, "uniform"), (6, 8192, 3, "normal")])
+def test_quantizer_variants_match_oracle(amq, rows, n, k, dist, method, final_refit):
+    """Final coefficient refit and refined greedy (the comparison methods of Sec. 2) against the oracle's variants:
+    rows whose codes agree must agree in the coefficients (1e-4 relative); rows whose codes differ (an element on a
+    decision boundary in fp32) must be rare and reach the same error within 1e-3."""
+    x = draw(dist, (rows, n), 300 + n + k)
+    g_codes, g_coeffs = amq.quantize_variant(dev(x), k, 2, method, final_refit)
+    g_codes, g_coeffs = codes_np(g_codes), g_coeffs.cpu().numpy().astype(np.float64)
+    assert parity.pad_bits_zero(g_codes, n)
+    o_codes, o_coeffs = oracle.quantize_rows_variant(x.astype(np.float64), k, 2, method, final_refit)
+    gb, ob = parity.unpack_rows(g_codes, n), parity.unpack_rows(o_codes, n)
+    differing = 0
+    for r in range(rows):
+        w = x[r].astype(np.float64)
+        if np.array_equal(gb[r], ob[r]):
+            assert np.abs(g_coeffs[r] - o_coeffs[r]).max() <= parity.COEFF_REL * np.abs(o_coeffs[r]).max() + 1e-30, r
+        else:
+            differing += 1
+            og, oo = oracle.objective(w, g_coeffs[r], gb[r]), oracle.objective(w, o_coeffs[r], ob[r])
+            assert abs(og - oo) <= 1e-3 * max(oo, 1e-30) + 1e-12 * (w ** 2).sum(), (r, og, oo)
+    assert differing <= max(2, 0.05 * rows), differing
+    if method == 0:
+        # the codes of the final-refit variant are those of the production kernel (Algorithm 2 as printed)
+        p_codes, _ = amq.quantize(dev(x), k, 2)
+        same = (codes_np(p_codes) == g_codes).all(axis=(1, 2)).sum()
+        assert same >= rows - max(2, 0.05 * rows)
+
+
+def test_error_ordering_of_the_methods_on_the_device(amq):
+    """Tables 1-2 order the methods by quantization error: greedy >= refined greedy >= alternating; a last coefficient
+    refit can only lower the error further.  Checked on the library's own results (mean relative MSE over 64 rows)."""
+    x = dev(draw("normal", (64, 1024), 900))
+    norm = (x.double() ** 2).sum()
+    for k in (2, 3, 4):
+        err = {}
+        for label, T, method, final in (("greedy", 0, 0, False), ("refined", 0, 1, False), ("alternating", 2, 0, False),
+                                        ("alternating+refit", 2, 0, True)):
+            codes, coeffs = amq.quantize_variant(x, k, T, method, final)
+            err[label] = float(((x.double() - amq.unpack(codes, coeffs, 1024).double()) ** 2).sum() / norm)
+        print(k, err)
+        assert err["greedy"] >= err["refined"] >= err["alternating"] >= err["alternating+refit"] > 0
