@@ -55,6 +55,7 @@ _lstm_paper = _sig("amq_oracle_lstm_step_paper", None, _u32p, _dp, _u32p, _dp, _
                    _dp, _dp, _int, _int, _int, _dp, _dp)
 _lsm = _sig("amq_oracle_log_softmax_argmax", None, _dp, _int, _int, _dp, _i32p)
 _gru = _sig("amq_oracle_gru_step", None, _u32p, _dp, _dp, _int, _int, _int, _dp, _dp, _int, _int, _int, _dp)
+_gru_orig = _sig("amq_oracle_gru_step_original", None, _u32p, _dp, _dp, _int, _int, _int, _dp, _dp, _int, _int, _int, _dp)
 _lstm_seq = _sig("amq_oracle_lstm_sequence", None, _u32p, _dp, _dp, _int, _int, _int, _dp, _int, _dp, _dp,
                  _int, _int, _int, _dp, _dp, _dp)
 _gru_seq = _sig("amq_oracle_gru_sequence", None, _u32p, _dp, _dp, _int, _int, _int, _dp, _int, _dp,
@@ -277,6 +278,17 @@ def gru_step(Wcodes, Walpha, bias, I, H, x, h, k_a, T):
     h_out = np.zeros((batch, H))
     _gru(_p(Wc, _u32p), _p(Wa, _dp), _p(bias, _dp), I, H, k_w, _p(x, _dp), _p(h, _dp),
          batch, k_a, T, _p(h_out, _dp))
+    return h_out
+
+
+def gru_step_original(Wcodes, Walpha, bias, I, H, x, h, k_a, T):
+    """The GRU in its original form (reset gate applied to h before the candidate's product; bias (3H,) or None)."""
+    Wc = np.ascontiguousarray(Wcodes, dtype=np.uint32)
+    Wa, x, h = _d(Walpha), _d(x), _d(h)
+    batch, k_w = x.shape[0], Wc.shape[1]
+    bias = None if bias is None else _d(bias)
+    h_out = np.zeros((batch, H))
+    _gru_orig(_p(Wc, _u32p), _p(Wa, _dp), _p(bias, _dp), I, H, k_w, _p(x, _dp), _p(h, _dp), batch, k_a, T, _p(h_out, _dp))
     return h_out
 
 

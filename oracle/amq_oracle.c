@@ -464,6 +464,41 @@ void amq_oracle_gru_step(const uint32_t* Wcodes, const double* Walpha, const dou
 }
 
 /* ---------------------------------------------------------------------------------------------
+ * One quantized GRU step in the original form of the GRU the paper cites (Cho et al., 2014): the reset gate
+ * multiplies the previous state BEFORE the candidate's product, so the step quantizes two vectors on-line:
+ *   z1 = [x ; h]:      r = logistic(W_r z1_hat + b_r),  z = logistic(W_z z1_hat + b_z);
+ *   z2 = [x ; r * h]:  cand = tanh(W_n z2_hat + b_n);   h' = (1 - z) * cand + z * h.
+ * W: 3H rows in the order r, z, n over n = I + H columns; bias has 3H entries [b_r; b_z; b_n] or is NULL.
+ * ------------------------------------------------------------------------------------------- */
+void amq_oracle_gru_step_original(const uint32_t* Wcodes, const double* Walpha, const double* bias,
+                                  int I, int H, int k_w, const double* x, const double* h_in,
+                                  int batch, int k_a, int T, double* h_out)
+{
+    int n = I + H, wpr = amq_oracle_words_per_row(n);
+    double* z = (double*)malloc(sizeof(double) * (size_t)n);
+    double* p = (double*)malloc(sizeof(double) * (size_t)3 * H);
+    double* pn = (double*)malloc(sizeof(double) * (size_t)H);
+    uint32_t* zc = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)k_a * wpr);
+    double beta[AMQ_ORACLE_MAX_K];
+    for (int bt = 0; bt < batch; ++bt) {
+        const double* h = h_in + (size_t)bt * H;
+        for (int t = 0; t < I; ++t) z[t] = x[(size_t)bt * I + t];
+        for (int t = 0; t < H; ++t) z[I + t] = h[t];
+        amq_oracle_quantize_rows(z, 1, n, n, k_a, T, zc, beta);
+        amq_oracle_binary_gemm(Wcodes, Walpha, 2 * H, n, k_w, zc, beta, 1, k_a, bias, p);      /* rows r, z */
+        for (int u = 0; u < H; ++u) z[I + u] = logistic(p[u]) * h[u];                          /* r * h */
+        amq_oracle_quantize_rows(z, 1, n, n, k_a, T, zc, beta);
+        amq_oracle_binary_gemm(Wcodes + (size_t)2 * H * k_w * wpr, Walpha + (size_t)2 * H * k_w, H, n, k_w,
+                               zc, beta, 1, k_a, bias ? bias + 2 * H : NULL, pn);               /* rows n */
+        for (int u = 0; u < H; ++u) {
+            double zg = logistic(p[H + u]);
+            h_out[(size_t)bt * H + u] = (1.0 - zg) * tanh(pn[u]) + zg * h[u];
+        }
+    }
+    free(z); free(p); free(pn); free(zc);
+}
+
+/* ---------------------------------------------------------------------------------------------
  * Output layer of Eq. 6: y = softmax(W_s h + b_s), stated here on given logits: log-probabilities
  * logp[t] = z[t] - max - log(sum_u exp(z[u] - max)) and the index of the largest logit (the first
  * one among equal maxima).  Plain definition, fp64.

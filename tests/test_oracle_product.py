@@ -269,3 +269,58 @@ def test_log_softmax_argmax_against_library_routine_and_invariants():
     assert np.array_equal(arg, z.argmax(axis=1)) and arg[1] == 17
     shifted, _ = oracle.log_softmax_argmax(z + 5.0)             # invariant to a common shift
     assert np.allclose(shifted, logp, atol=1e-10)
+
+
+def textbook_gru_original(W, b, x, h, I, H):
+    """Cho et al.: r, z from [x ; h]; candidate from [x ; r * h]; W rows r, z, n; b (3H,) or None."""
+    sig = lambda v: 1 / (1 + np.exp(-v))
+    b = np.zeros(3 * H) if b is None else b
+    zcat = np.concatenate([x, h], axis=1)
+    r = sig(zcat @ W[:H].T + b[:H])
+    z = sig(zcat @ W[H:2 * H].T + b[H:2 * H])
+    cand = np.tanh(np.concatenate([x, r * h], axis=1) @ W[2 * H:].T + b[2 * H:])
+    return (1 - z) * cand + z * h
+
+
+@pytest.mark.parametrize("I,H,batch,kw,ka", [(20, 12, 2, 2, 3), (33, 31, 1, 3, 3), (37, 40, 3, 2, 2)])
+def test_original_form_gru_equals_textbook_step_on_reconstructed_operands(I, H, batch, kw, ka):
+    """The composition: both on-line quantizations and both products, checked against dense fp64 algebra on the
+    reconstructed operands (the second vector depends on the first product through r)."""
+    n = I + H
+    W = synth.normal((3 * H, n), 0.2, 28, 1).astype(np.float64)
+    bias = synth.normal((3 * H,), 0.1, 28, 2).astype(np.float64)
+    x = synth.normal((batch, I), 1.0, 28, 3).astype(np.float64)
+    h = synth.uniform((batch, H), -1, 1, 28, 4).astype(np.float64)
+    Wc, Wa = oracle.quantize_rows(W, kw, 2)
+    What = dense_hat(Wc, Wa, n)
+    sig = lambda v: 1 / (1 + np.exp(-v))
+    z1c, z1b = oracle.quantize_rows(np.concatenate([x, h], axis=1), ka, 2)
+    z1 = dense_hat(z1c, z1b, n)
+    r = sig(z1 @ What[:H].T + bias[:H])
+    zg = sig(z1 @ What[H:2 * H].T + bias[H:2 * H])
+    z2c, z2b = oracle.quantize_rows(np.concatenate([x, r * h], axis=1), ka, 2)
+    cand = np.tanh(dense_hat(z2c, z2b, n) @ What[2 * H:].T + bias[2 * H:])
+    ref = (1 - zg) * cand + zg * h
+    got = oracle.gru_step_original(Wc, Wa, bias, I, H, x, h, ka, 2)
+    assert np.allclose(got, ref, rtol=1e-11, atol=1e-13)
+    assert np.array_equal(oracle.gru_step_original(Wc, Wa, None, I, H, x, h, ka, 2),
+                          oracle.gru_step_original(Wc, Wa, np.zeros(3 * H), I, H, x, h, ka, 2))
+
+
+def test_original_form_gru_reduces_to_the_textbook_gru_when_quantization_is_the_identity():
+    # [x ; h] takes values in {+-a +-c} (2 bits exact); with W_r = 0 and b_r large the reset gate is 1 to 1e-16, so
+    # [x ; r * h] is exactly representable too and the quantized step must equal the plain fp64 step of Cho et al.
+    I, H, batch = 24, 16, 2
+    n = I + H
+    z = exactly_representable((batch, n), 0.5, 0.125, 29, 1)
+    x, h = z[:, :I], z[:, I:]
+    W = exactly_representable((3 * H, n), 0.05, 0.02, 29, 2)
+    W[:H] = 0.0
+    bias = np.concatenate([np.full(H, 40.0), synth.normal((2 * H,), 0.1, 29, 3).astype(np.float64)])
+    Wc, Wa = oracle.quantize_rows(W, 2, 2)
+    got = oracle.gru_step_original(Wc, Wa, bias, I, H, x, h, 2, 2)
+    assert np.allclose(got, textbook_gru_original(W, bias, x, h, I, H), atol=1e-12)
+    # and it differs from the linear-before-reset form as soon as r is not 1 (the two forms are different cells)
+    bias2 = bias.copy(); bias2[:H] = 0.0
+    a = oracle.gru_step_original(Wc, Wa, bias2, I, H, x, h, 2, 2)
+    assert np.abs(a - got).max() > 1e-3
