@@ -219,6 +219,20 @@ AMQ_API amq_status amq_gru_sequence(const uint32_t* Wcodes, const float* Walpha,
                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * GRU step in the original form of the GRU the paper cites (Cho et al., 2014; the paper prints no GRU equations):
+ *   z1 = [x ; h] quantized on-line:      r = logistic(W_r z1_hat + b_r),  z = logistic(W_z z1_hat + b_z);
+ *   z2 = [x ; r * h] quantized on-line:  cand = tanh(W_n z2_hat + b_n);   h' = (1 - z) * cand + z * h.
+ * Wcodes / Walpha as for amq_gru_step (3H rows r, z, n over I + H columns); bias [3H] = [b_r; b_z; b_n] or NULL;
+ * x [batch][I], h_in / h_out [batch][H] DEVICE fp32, h_out != h_in; workspace: DEVICE,
+ * amq_gru_original_workspace_bytes(...) bytes, 16-byte aligned.  Two quantizations and two products per step
+ * (amq_gru_step, which applies r after the product, needs one of each).  Errors as amq_gru_step.
+ */
+AMQ_API size_t amq_gru_original_workspace_bytes(int I, int H, int batch, int k_a);
+AMQ_API amq_status amq_gru_step_original(const uint32_t* Wcodes, const float* Walpha, const float* bias, int I, int H, int k_w,
+                                 const float* x, const float* h_in, int batch, int k_a, int T, float* h_out,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The LSTM in the form the paper states it (Eq. 6 and the paragraph after it): separate matrices W_i (4H x I)
  * and W_h (4H x H), each quantized row by row; x_t is a row of the quantized embedding matrix and needs no
  * further quantization; only h_{t-1} is quantized on-line.

@@ -52,6 +52,8 @@ EXPORTS = {
     "amq_gru_sequence_host": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _int, _vp, _int, _int, _int,
                                      _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
     "amq_workspace_status": (_int, [_vp, _vp]),
+    "amq_gru_original_workspace_bytes": (_sz, [_int, _int, _int, _int]),
+    "amq_gru_step_original": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _vp, _int, _int, _int, _vp, _vp, _sz, _vp]),
     "amq_quantize_variant": (_int, [_vp, _int, _int, _int, _int, _int, _int, _int, _vp, _vp, _vp]),
     "amq_lm_decode_workspace_bytes": (_sz, [_int, _int, _int, _int, _int]),
     "amq_lm_greedy_decode": (_int, [_vp, _vp, _int, _int, _int, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp, _vp, _vp, _int,
@@ -384,3 +386,14 @@ def quantize_variant(x, k, T, method=METHOD_ALTERNATING, final_refit=False):
     _check(_lib.amq_quantize_variant(_ptr(x), rows, n, ldx, k, T, method, int(final_refit), _ptr(codes), _ptr(coeffs),
                                      _stream()))
     return codes, coeffs
+
+
+def gru_step_original(Wcodes, Walpha, bias, I, H, x, h_in, k_a, T, workspace=None, h_out=None):
+    """The GRU in its original form (reset gate applied to h before the candidate's product); bias (3H,) or None."""
+    batch, k_w = h_in.shape[0], Wcodes.shape[1]
+    if workspace is None:
+        workspace = torch.empty((_lib.amq_gru_original_workspace_bytes(I, H, batch, k_a),), dtype=torch.uint8, device=h_in.device)
+    h_out = torch.empty_like(h_in) if h_out is None else h_out
+    _check(_lib.amq_gru_step_original(_ptr(Wcodes), _ptr(Walpha), _ptr(bias), I, H, k_w, _ptr(x), _ptr(h_in), batch, k_a, T,
+                                      _ptr(h_out), _ptr(workspace), workspace.numel(), _stream()))
+    return h_out

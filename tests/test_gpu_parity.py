@@ -392,3 +392,28 @@ def test_error_ordering_of_the_methods_on_the_device(amq):
             err[label] = float(((x.double() - amq.unpack(codes, coeffs, 1024).double()) ** 2).sum() / norm)
         print(k, err)
         assert err["greedy"] >= err["refined"] >= err["alternating"] >= err["alternating+refit"] > 0
+
+
+@pytest.mark.parametrize("I,H,kw,ka,batch", [(64, 40, 2, 3, 19), (100, 129, 3, 2, 5), (33, 31, 1, 4, 1), (256, 512, 2, 2, 64),
+                                             (0, 48, 2, 2, 3)])
+def test_gru_step_in_the_original_form_matches_oracle(amq, I, H, kw, ka, batch):
+    """Cho et al.'s GRU: two on-line quantizations per step, the second on [x ; r * h].  The step is compared as a
+    whole (the second vector depends on the first product) within the state tolerance, with and without bias, and
+    chained for three steps teacher-forced on the oracle's state."""
+    n = I + H
+    Wc, Wa, _ = cell_setup("gru", I, H, kw, 60 + H, 0.05)
+    bias = synth.normal((3 * H,), 0.1, 61, 5)
+    x = synth.uniform((batch, I), -1, 1, 61, 1)
+    h = synth.uniform((batch, H), -1, 1, 61, 2)
+    dWc, dWa = codes_dev(Wc), dev(Wa, torch.float32)
+    for step in range(3):
+        _, beta = oracle.quantize_rows(np.concatenate([x, h], axis=1).astype(np.float64), ka, 2)
+        tol = state_tolerance(Wa, beta, n)
+        h_ref = oracle.gru_step_original(Wc, Wa, bias, I, H, x, h, ka, 2)
+        h_out = amq.gru_step_original(dWc, dWa, dev(bias), I, H, dev(x), dev(h), ka, 2)
+        assert np.abs(h_out.cpu().numpy() - h_ref).max() <= tol, step
+        h_nb = amq.gru_step_original(dWc, dWa, None, I, H, dev(x), dev(h), ka, 2)
+        assert np.abs(h_nb.cpu().numpy() - oracle.gru_step_original(Wc, Wa, None, I, H, x, h, ka, 2)).max() <= tol
+        h = h_ref.astype(np.float32)
+        x = synth.uniform((batch, I), -1, 1, 62 + step, 1)
+    assert amq.device_status() == 0
