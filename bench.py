@@ -572,9 +572,23 @@ def table6_lines(amq, torch, dev, flush):
                 run()
             cold = _event_ms(torch, run, flush, 10)
             warm = _burst_ms(torch, run, 50)
-            out.append({"workload": "Table 6 shape: quantize(h) + binary product %d x %d, %d/%d bits, batch 1" % (m, n, k, k),
-                        "ms_cold": cold, "ms_warm": warm, "bound": "latency (two launches)",
-                        "paper_cpu_ms_one_xeon_core": paper_ms[(m, k)]})
+            line = {"workload": "Table 6 shape: quantize(h) + binary product %d x %d, %d/%d bits, batch 1" % (m, n, k, k),
+                    "ms_cold": cold, "ms_warm": warm, "bound": "latency (two launches)",
+                    "paper_cpu_ms_one_xeon_core": paper_ms[(m, k)]}
+            try:
+                # the same two launches replayed from a CUDA graph: device time without the cost of the Python calls
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    run()
+                    with torch.cuda.graph(graph, stream=side):
+                        run()
+                torch.cuda.current_stream().wait_stream(side)
+                line["ms_warm_graph_replay"] = _burst_ms(torch, graph.replay, 50)
+            except Exception as exc:                                  # the line stays without the replay figure
+                line["graph_replay_error"] = str(exc)[:120]
+            out.append(line)
             del Wc, Wa
     return out
 
@@ -622,12 +636,29 @@ def greedy_decoding_line(amq, torch, dev):
     tokens = torch.zeros((ntok + 1,), dtype=torch.int32, device=dev)
     h, c = torch.zeros((1, H), device=dev), torch.zeros((1, H), device=dev)
 
+    first = torch.tensor([17], dtype=torch.int32, device=dev)
+
     def run():
-        tokens[0] = 17
+        tokens[0:1].copy_(first)
         amq.lm_greedy_decode(Wec, Wea, Wic, Wia, Whc, Wha, None, Wsc, Wsa, bs, I, H, k, 2, tokens, h, c, ws)
 
     ms = _burst_ms(torch, run, 5)
-    return {"workload": "greedy decoding, vocabulary %d, I=H=%d, 2/2 bits, one sequence, %d tokens per call (embedding row, "
+    extra = {}
+    try:
+        # the same chain (7 launches per token) captured once in a CUDA graph and replayed
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            run()
+            with torch.cuda.graph(graph, stream=side):
+                run()
+        torch.cuda.current_stream().wait_stream(side)
+        gms = _burst_ms(torch, graph.replay, 5)
+        extra = {"us_per_token_graph_replay": 1e3 * gms / ntok, "tokens_per_s_graph_replay": ntok * 1e3 / gms}
+    except Exception as exc:
+        extra = {"graph_replay_error": str(exc)[:120]}
+    return {**extra, "workload": "greedy decoding, vocabulary %d, I=H=%d, 2/2 bits, one sequence, %d tokens per call (embedding row, "
                         "paper-form cell, quantize(h), output product, log-softmax/arg-max; token fed back on the device)" % (
                             V, H, ntok),
             "ms": ms, "bound": "latency", "us_per_token": 1e3 * ms / ntok, "tokens_per_s": ntok * 1e3 / ms,

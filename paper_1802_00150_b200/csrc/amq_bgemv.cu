@@ -205,7 +205,7 @@ amq_status launch_cfg(const GemvParams& p, cudaStream_t st)
     }
     constexpr int PASSES = SEG / R;
     const long long passes = ((long long)p.m + 31) / 32 * PASSES;
-    const long long need = (passes + 31) / 32;                          // at least four passes per warp
+    const long long need = (passes + 7) / 8;                            // small matrices: one pass per warp, spread over the SMs
     const int limit = cached_grid[exact ? 1 : 0];
     const int grid = (int)(need < limit ? need : limit);
     kernel<<<grid, 256, 0, st>>>(p);
