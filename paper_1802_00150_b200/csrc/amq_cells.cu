@@ -34,7 +34,8 @@ amq_status enqueue_persistent(const CellCall& c, const CellWorkspace& ws, const 
                               const float* h0, const float* c0, float* h_seq, float* h_last, float* c_last,
                               cudaStream_t st)
 {
-    AMQ_CUDA_TRY(cudaMemsetAsync(ws.hx, 0, (size_t)2 * c.H * 8, st));     // stale step tags must not match
+    if (steps > 1)      // stale step tags must not match (a single step polls nothing)
+        AMQ_CUDA_TRY(cudaMemsetAsync(ws.hx, 0, (size_t)2 * c.H * 8, st));
     return launch_rnn_persistent(c.Wcodes, c.Walpha, c.bias, c.I, c.H, c.k_w, c.k_a, c.T, c.gru, x_seq, steps,
                                  h0, c0, h_seq, h_last, c_last, ws.hx, ws.status, st);
 }

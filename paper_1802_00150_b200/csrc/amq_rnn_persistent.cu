@@ -319,6 +319,12 @@ amq_status launch(const PersistArgs& a, int grid, size_t smem, cudaStream_t st)
     AMQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     PersistArgs args = a;
     void* params[] = {&args};
+    if (a.steps <= 1) {
+        // a single step never waits for another CTA (step 0 reads h0): a plain launch is enough and cheaper
+        kernel<<<dim3((unsigned)grid), dim3(NT), smem, st>>>(args);
+        AMQ_LAUNCH_CHECK();
+        return AMQ_OK;
+    }
     AMQ_CUDA_TRY(cudaLaunchCooperativeKernel((void*)kernel, dim3((unsigned)grid), dim3(NT), params, smem, st));
     __atomic_fetch_add(&g_kernel_launches, 1ull, __ATOMIC_RELAXED);
     return AMQ_OK;
