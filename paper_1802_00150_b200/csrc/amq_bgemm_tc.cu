@@ -193,6 +193,15 @@ __device__ __forceinline__ float small_int_to_float(int v)
     return __int_as_float(v + 0x4B400000) - 12582912.0f;
 }
 
+// Loads of what the preceding kernel of the stream may have produced (activation planes, their coefficients, added
+// pre-activations) are ordinary L2-cached loads (__ldcg), not read-only-path loads: with an overlapped launch this
+// kernel is alive while those bytes are still being written, and a read-only load may be moved above the wait.
+
+__device__ __forceinline__ uint4 load_row_chunk(const uint4* p, bool weight_row)
+{
+    return weight_row ? __ldg(p) : __ldcg(p);       // weights are constant; activation planes: see above
+}
+
 // one 128-bit chunk of a packed row -> its 128 operand bytes (eight 16-byte pieces at the swizzled offsets `off`)
 __device__ __forceinline__ void expand_chunk(uint32_t base, const uint32_t (&off)[8], const uint4& v, const uint32_t (&mul)[7],
                                              uint32_t m_sign, uint32_t m_half)
@@ -342,7 +351,7 @@ __device__ __forceinline__ void epilogue_smem_to_global(const TcParams& p, const
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     float s = bias4[g];
-                    if (a.addend) s += __ldg(a.addend + (size_t)(b0 + bb) * a.ld_addend + g * H + u);
+                    if (a.addend) s += __ldcg(a.addend + (size_t)(b0 + bb) * a.ld_addend + g * H + u);
                     for (int i = 0; i < k_w; ++i) s += y0[(g * k_w + i) * ldy + bb];
                     g4[g] = s;
                 }
@@ -476,15 +485,20 @@ bgemm_tc_kernel(TcParams p)
         const uint32_t m_sign = p.mask_sign, m_half = p.mask_half;  // 0x80808080, 0x40404040
         const uint4 zero = make_uint4(0, 0, 0, 0);
 
-        uint4 cur = (src && grp < CH) ? __ldg(src + grp) : zero;    // own steps: grp, grp + G, ..
-        uint4 nxt = (src && grp + G < CH) ? __ldg(src + grp + G) : zero;
+        // weight rows are fetched at once; everything the preceding kernel of the stream may have written (the
+        // activation planes and their coefficients, the state) is read after the wait
+        const bool weight_row = r_all < MT * TILE_M;
+        if (!weight_row) grid_dependency_wait();
+        uint4 cur = (src && grp < CH) ? load_row_chunk(src + grp, weight_row) : zero;       // own steps: grp, grp + G, ..
+        uint4 nxt = (src && grp + G < CH) ? load_row_chunk(src + grp + G, weight_row) : zero;
+        if (weight_row) grid_dependency_wait();
         // coefficients for the epilogue, after the first operand loads are under way (the stores below wait for
         // their loads; the latency hides behind the main loop)
         if (coef_dst) {
-            *coef_dst = coef_src ? __ldg(coef_src) : 0.0f;
+            *coef_dst = coef_src ? __ldcg(coef_src) : 0.0f;
             if (r_all >= MT * TILE_M && (r_all - MT * TILE_M) % KA == 0) {
                 float sum = 0.0f;
-                for (int jj = 0; jj < KA; ++jj) sum += corr_src ? __ldg(corr_src + jj) : 0.0f;
+                for (int jj = 0; jj < KA; ++jj) sum += corr_src ? __ldcg(corr_src + jj) : 0.0f;
                 sBcorr[(r_all - MT * TILE_M) / KA] = -(float)(p.wpr * 32 - a.n) * sum;
             }
         }
@@ -493,7 +507,7 @@ bgemm_tc_kernel(TcParams p)
         for (int c = grp; c < CH; c += G) {
             const uint4 v = cur;
             cur = nxt;
-            nxt = (src && c + 2 * G < CH) ? __ldg(src + c + 2 * G) : zero;
+            nxt = (src && c + 2 * G < CH) ? load_row_chunk(src + c + 2 * G, weight_row) : zero;
             // the MMAs that read this buffer one lap ago must have completed
             if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; break; }
             if (writes) {
@@ -667,13 +681,15 @@ bgemm_tc_persistent_kernel(TcParams p)
         const uint4* pf_src = row_of(pf_tile);
         auto pf_load = [&]() -> uint4 {
             while (pf_c >= CH) { pf_c -= CH; pf_tile += tile_step; pf_src = row_of(pf_tile); }
-            const uint4 v = pf_src ? __ldg(pf_src + pf_c) : zero;
+            const uint4 v = pf_src ? load_row_chunk(pf_src + pf_c, is_a) : zero;
             pf_c += G;
             return v;
         };
         const int my_tiles = (ntiles - (int)blockIdx.x + tile_step - 1) / tile_step;
         const int total = my_tiles * CH;
+        if (!is_a) grid_dependency_wait();                          // activation planes come from the preceding kernel
         uint4 cur = pf_load(), nxt = pf_load();
+        if (is_a) grid_dependency_wait();
         int buf = grp;                                              // G <= S
         uint32_t empty_parity = 1;
         for (int q = grp; q < total; q += G) {
@@ -728,6 +744,7 @@ bgemm_tc_persistent_kernel(TcParams p)
         // ---- epilogue warps ----
         const int tid_e = tid - epi_warp0 * 32, nth_e = EW * 32;
         const int quarter = warp & 3, slot = (warp - epi_warp0) >> 2, nslots = EW >> 2;
+        grid_dependency_wait();                                     // coefficients and state come from preceding kernels
         int it = 0;
         for (int tile = (int)blockIdx.x; tile < ntiles; tile += tile_step, ++it) {
             const int ab = (p.nbuf == 2) ? (it & 1) : 0;
@@ -745,10 +762,10 @@ bgemm_tc_persistent_kernel(TcParams p)
                 for (int idx = tid_e; idx < n_mma; idx += nth_e) {
                     const int e = idx / KA, j = idx - e * KA, b = b0 + e;
                     const bool use_b = b < a.batch;
-                    sBeta[idx] = use_b ? __ldg(a.xbeta + (size_t)b * KA + j) : 0.0f;
+                    sBeta[idx] = use_b ? __ldcg(a.xbeta + (size_t)b * KA + j) : 0.0f;
                     if (j == 0) {
                         float sum = 0.0f;
-                        for (int jj = 0; jj < KA; ++jj) sum += use_b ? __ldg(a.xbeta + (size_t)b * KA + jj) : 0.0f;
+                        for (int jj = 0; jj < KA; ++jj) sum += use_b ? __ldcg(a.xbeta + (size_t)b * KA + jj) : 0.0f;
                         sBcorr[e] = -(float)(p.wpr * 32 - a.n) * sum;
                     }
                 }
@@ -898,6 +915,17 @@ amq_status launch_ka(const TcPlan& pl, cudaStream_t st)
 {
     auto kernel = pl.persistent ? bgemm_tc_persistent_kernel<KA> : bgemm_tc_kernel<KA>;
     AMQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+    if (pl.p.a.overlap_with_previous) {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = pl.grid; cfg.blockDim = dim3((unsigned)pl.threads); cfg.dynamicSmemBytes = pl.smem; cfg.stream = st;
+        cudaLaunchAttribute attr{};
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr; cfg.numAttrs = 1;
+        AMQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, kernel, pl.p));
+        AMQ_LAUNCH_CHECK();
+        return AMQ_OK;
+    }
     kernel<<<pl.grid, pl.threads, pl.smem, st>>>(pl.p);
     AMQ_LAUNCH_CHECK();
     return AMQ_OK;

@@ -68,6 +68,7 @@ amq_status enqueue_step(const CellCall& c, const CellWorkspace& ws, const float*
     if (s != AMQ_OK) return s;
     a.epilogue = c.gru ? EPI_GRU : EPI_LSTM;
     a.I = c.I; a.H = c.H; a.h_in = h_in; a.c_in = c_in; a.h_out = h_out; a.c_out = c_out;
+    a.overlap_with_previous = true;             // the quantizer above is the previous kernel of the stream
     return launch_binary_gemm(a, st);
 }
 

@@ -88,6 +88,7 @@ amq_status recurrent_part(const PaperCall& c, const PaperWorkspace& ws, const fl
     }
     a.y = nullptr; a.ldy = 0;
     a.epilogue = EPI_LSTM;
+    a.overlap_with_previous = true;             // the quantizer above is the previous kernel of the stream
     a.I = 0; a.H = c.H; a.h_in = h_in; a.c_in = c_in; a.h_out = h_out; a.c_out = c_out;
     a.addend = proj; a.ld_addend = 4 * c.H;
     return launch_binary_gemm(a, st);

@@ -87,7 +87,16 @@ struct GemmArgs {
     // EPI_LSTM only: optional pre-activations computed elsewhere (e.g. W_i x), added before the gates;
     // addend[b * ld_addend + gate * H + unit]
     const float* addend; int ld_addend;
+    // the launch may start while the previous kernel of the stream (the on-line quantizer that produces xcodes / xbeta)
+    // still runs: the kernel sets itself up, fetches weights, and waits for that kernel before it reads anything else
+    bool overlap_with_previous;
 };
+
+// programmatic dependent launch (sm_90+): `grid_dependency_wait` returns once the preceding kernel of the stream has
+// completed and its writes are visible (at once when the launch was an ordinary one); `grid_dependents_may_launch`
+// lets the next kernel's CTAs be scheduled early (a no-op when that launch does not ask for it)
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st);
 

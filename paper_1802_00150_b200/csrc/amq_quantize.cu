@@ -69,6 +69,7 @@ __global__ void __launch_bounds__(256)
 quantize_kernel(RowSource src, int rows, int n, int T, uint32_t* __restrict__ codes, float* __restrict__ coeffs)
 {
     __shared__ QuantScratch<K> scratch[MULTI ? 1 : 4];
+    grid_dependents_may_launch();       // the product kernel that follows may set itself up while this one runs
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = MULTI ? blockDim.x : 32;

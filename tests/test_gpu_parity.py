@@ -417,3 +417,27 @@ def test_gru_step_in_the_original_form_matches_oracle(amq, I, H, kw, ka, batch):
         h = h_ref.astype(np.float32)
         x = synth.uniform((batch, I), -1, 1, 62 + step, 1)
     assert amq.device_status() == 0
+
+
+@pytest.mark.parametrize("cell,I,H,kw,ka,batch,steps", [("lstm", 256, 256, 2, 2, 20, 6), ("gru", 256, 192, 2, 3, 33, 5)])
+def test_batched_sequences_repeat_bit_for_bit(amq, cell, I, H, kw, ka, batch, steps):
+    """The product kernel of a timestep is launched so that it may start while the quantizer of that timestep still
+    runs (it waits for it before reading the planes).  A read that slipped ahead of that wait would show up as results
+    that change from run to run: five runs of the same sequence must agree bit for bit."""
+    Wc, Wa, bias = cell_setup(cell, I, H, kw, 70 + H, 0.08)
+    xs = dev(synth.normal((steps, batch, I), 1.0, 71, 1))
+    h0 = dev(synth.uniform((batch, H), -1, 1, 71, 2))
+    c0 = dev(synth.uniform((batch, H), -1, 1, 71, 3))
+    ws = amq.new_workspace(I, H, batch, ka)
+    dWc, dWa, dbias = codes_dev(Wc), dev(Wa, torch.float32), dev(bias)
+    runs = []
+    for _ in range(5):
+        if cell == "lstm":
+            seq, _, _ = amq.lstm_sequence(dWc, dWa, dbias, I, H, xs, h0, c0, ka, 2, ws, want_h_seq=True)
+        else:
+            seq, _ = amq.gru_sequence(dWc, dWa, dbias, I, H, xs, h0, ka, 2, ws, want_h_seq=True)
+        runs.append(seq.clone())
+        junk = torch.rand((batch, ka), device="cuda")          # other traffic between the runs
+        del junk
+    for r in runs[1:]:
+        assert torch.equal(r, runs[0])
