@@ -942,6 +942,13 @@ bool gemm_tc_supported(const GemmArgs& a)
     return (a.batch >= 16 || (a.batch >= 2 && big)) && plan(a, &pl);
 }
 
+bool gemm_tc_single_wave(const GemmArgs& a)
+{
+    TcPlan pl;
+    if (!gemm_tc_supported(a) || !plan(a, &pl)) return false;
+    return pl.persistent || (long long)pl.grid.x * pl.grid.y <= sm_count();
+}
+
 amq_status launch_binary_gemm_tc(const GemmArgs& a, cudaStream_t st)
 {
     TcPlan pl;

@@ -64,10 +64,13 @@ amq_status enqueue_step(const CellCall& c, const CellWorkspace& ws, const float*
     a.bias = c.bias;
     if (use_persistent(c))      // batch 1: one launch of the weight-stationary kernel, a sequence of one step
         return enqueue_persistent(c, ws, x, 1, h_in, c_in, nullptr, h_out, c_out, st);
-    amq_status s = launch_quantize(x, c.I, c.I, h_in, c.H, c.H, c.batch, c.k_a, c.T, ws.zcodes, ws.zbeta, st);
-    if (s != AMQ_OK) return s;
     a.epilogue = c.gru ? EPI_GRU : EPI_LSTM;
     a.I = c.I; a.H = c.H; a.h_in = h_in; a.c_in = c_in; a.h_out = h_out; a.c_out = c_out;
+    // the quantizer may be scheduled while the product of the previous timestep still runs (it waits for it first
+    // thing) when that product runs as a single wave
+    amq_status s = launch_quantize(x, c.I, c.I, h_in, c.H, c.H, c.batch, c.k_a, c.T, ws.zcodes, ws.zbeta, st,
+                                   gemm_tc_single_wave(a));
+    if (s != AMQ_OK) return s;
     a.overlap_with_previous = true;             // the quantizer above is the previous kernel of the stream
     return launch_binary_gemm(a, st);
 }

@@ -71,12 +71,16 @@ amq_status input_projection(const PaperCall& c, const uint32_t* xcodes, const fl
 amq_status recurrent_part(const PaperCall& c, const PaperWorkspace& ws, const float* proj, const float* h_in,
                           const float* c_in, float* h_out, float* c_out, cudaStream_t st)
 {
-    amq_status s = launch_quantize(h_in, c.H, c.H, nullptr, 0, 0, c.batch, c.k_a, c.T, ws.hcodes, ws.hbeta, st);
-    if (s != AMQ_OK) return s;
     GemmArgs a{};
     a.Wcodes = c.Wh_codes; a.Walpha = c.Wh_alpha; a.m = 4 * c.H; a.n = c.H; a.k_w = c.k_w;
     a.xcodes = ws.hcodes; a.xbeta = ws.hbeta; a.batch = c.batch; a.k_a = c.k_a;
     a.bias = nullptr;
+    a.epilogue = EPI_LSTM; a.H = c.H;
+    // in a sequence the kernel before this quantizer is the recurrent product of the previous timestep: when that
+    // runs as a single wave the quantizer may be scheduled behind it early (it waits for it first thing)
+    amq_status s = launch_quantize(h_in, c.H, c.H, nullptr, 0, 0, c.batch, c.k_a, c.T, ws.hcodes, ws.hbeta, st,
+                                   gemm_tc_single_wave(a));
+    if (s != AMQ_OK) return s;
     if (c.batch == 1) {
         // one sequence: the bandwidth-bound matrix-vector kernel writes the pre-activations, a small kernel applies the gates
         a.epilogue = EPI_Y; a.y = ws.gates; a.ldy = 4 * c.H;

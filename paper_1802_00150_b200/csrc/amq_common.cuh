@@ -68,7 +68,8 @@ inline CellWorkspace carve_cell_workspace(void* base, int I, int H, int batch, i
 
 // Quantize `rows` vectors; element t of row r is src0[r*ld0 + t] for t < n0, else src1[r*ld1 + t - n0].
 amq_status launch_quantize(const float* src0, int ld0, int n0, const float* src1, int ld1, int n1,
-                           int rows, int k, int T, uint32_t* codes, float* coeffs, cudaStream_t st);
+                           int rows, int k, int T, uint32_t* codes, float* coeffs, cudaStream_t st,
+                           bool overlap_with_previous = false);
 
 enum Epilogue { EPI_DOTS = 0, EPI_Y = 1, EPI_LSTM = 2, EPI_GRU = 3 };
 
@@ -92,13 +93,16 @@ struct GemmArgs {
     bool overlap_with_previous;
 };
 
-// programmatic dependent launch (sm_90+): `grid_dependency_wait` returns once the preceding kernel of the stream has
-// completed and its writes are visible (at once when the launch was an ordinary one); `grid_dependents_may_launch`
-// lets the next kernel's CTAs be scheduled early (a no-op when that launch does not ask for it)
+// programmatic dependent launch (sm_90+): a kernel launched with the programmatic-serialization attribute may have its
+// CTAs scheduled as the CTAs of the preceding kernel of the stream exit; `grid_dependency_wait` returns once that kernel
+// has completed and its writes are visible (at once when the launch was an ordinary one).  No kernel here signals
+// earlier than its exit: measured, early signals only made the waiting CTAs take SM resources sooner.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st);
+// whether the tensor-core kernel takes the problem with all its CTAs resident at once (then the quantizer of the next
+// timestep is launched as its programmatic dependent: its CTAs move in as the product's CTAs exit)
+bool gemm_tc_single_wave(const GemmArgs& a);
 
 // Batch-1 streaming kernel (EPI_DOTS / EPI_Y): whether it covers a problem, and its launch.
 // gates of Eq. 6 for one sequence from pre-activations pre[4H] (+ addend[4H] when given), rows i, f, o, g

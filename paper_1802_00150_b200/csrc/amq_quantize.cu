@@ -10,11 +10,13 @@ namespace {
 struct RowSource {
     const float* src0; int ld0; int n0;
     const float* src1; int ld1;
+    bool overlap_with_previous;     // host side only: launch as a programmatic dependent of the preceding kernel
 };
 
 __device__ __forceinline__ float load_elem(const RowSource& s, int row, int t)
 {
-    return (t < s.n0) ? __ldg(s.src0 + (size_t)row * s.ld0 + t) : __ldg(s.src1 + (size_t)row * s.ld1 + (t - s.n0));
+    // ordinary L2-cached loads: with an overlapped launch the state may still be written while this kernel is alive
+    return (t < s.n0) ? __ldcg(s.src0 + (size_t)row * s.ld0 + t) : __ldcg(s.src1 + (size_t)row * s.ld1 + (t - s.n0));
 }
 
 // Bulk variant, one row of up to 1024 elements per warp: lane l holds the 32 CONSECUTIVE elements 32 l ..
@@ -69,7 +71,7 @@ __global__ void __launch_bounds__(256)
 quantize_kernel(RowSource src, int rows, int n, int T, uint32_t* __restrict__ codes, float* __restrict__ coeffs)
 {
     __shared__ QuantScratch<K> scratch[MULTI ? 1 : 4];
-    grid_dependents_may_launch();       // the product kernel that follows may set itself up while this one runs
+    grid_dependency_wait();             // launched early behind a product kernel: its state output must be complete
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = MULTI ? blockDim.x : 32;
@@ -107,6 +109,18 @@ amq_status run(const RowSource& src, int rows, int n, int T, uint32_t* codes, fl
 {
     const int rows_per_cta = MULTI ? 1 : threads / 32;
     const unsigned grid = (unsigned)((rows + rows_per_cta - 1) / rows_per_cta);
+    if (src.overlap_with_previous) {
+        // may be scheduled while the preceding kernel of the stream still runs; the kernel waits for it first thing
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3((unsigned)threads); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute attr{};
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr; cfg.numAttrs = 1;
+        AMQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, quantize_kernel<K, EPT, MULTI>, src, rows, n, T, codes, coeffs));
+        AMQ_LAUNCH_CHECK();
+        return AMQ_OK;
+    }
     quantize_kernel<K, EPT, MULTI><<<grid, threads, 0, st>>>(src, rows, n, T, codes, coeffs);
     AMQ_LAUNCH_CHECK();
     return AMQ_OK;
@@ -136,9 +150,9 @@ amq_status dispatch(const RowSource& src, int rows, int n, int T, uint32_t* code
 }  // namespace
 
 amq_status launch_quantize(const float* src0, int ld0, int n0, const float* src1, int ld1, int n1,
-                           int rows, int k, int T, uint32_t* codes, float* coeffs, cudaStream_t st)
+                           int rows, int k, int T, uint32_t* codes, float* coeffs, cudaStream_t st, bool overlap_with_previous)
 {
-    RowSource src{src0, ld0, n0, src1, ld1};
+    RowSource src{src0, ld0, n0, src1, ld1, overlap_with_previous};
     const int n = n0 + n1;
     switch (k) {
         case 1: return dispatch<1>(src, rows, n, T, codes, coeffs, st);
