@@ -409,6 +409,7 @@ def run_ours(args, wl):
         }
         if not args.no_extras and world == 1:
             line["gemv_cold"] = cold_gemv(amq, torch, dev, flush, peak, peak_kind)
+            line["gemv_rotated"] = rotated_gemv(amq, torch, dev, peak, peak_kind)
             line["batched"] = batched_lines(amq, torch, dev, flush, peak, peak_kind)
             assert amq.device_status() == 0
         if not args.no_cpu_baseline and world == 1:
@@ -470,6 +471,49 @@ def cold_gemv(amq, torch, dev, flush, peak, peak_kind):
                     "ms": ms, "bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": peak, "frac": gbs / peak,
                     "peak_kind": "of " + peak_kind, "frac_of_nominal_8000": gbs / 8000.0, "algorithmic_bytes": int(alg)})
         del Wcodes, Walpha, y
+    return out
+
+
+def rotated_gemv(amq, torch, dev, peak, peak_kind):
+    """The small matrix-vector shapes (the two of Table 6 and 32768 x 1024) kept cold by rotating over distinct weight
+    copies that together exceed twice the L2: one launch per copy, the whole rotation replayed from a CUDA graph so that
+    the gaps between the launches are those of the device.  GB/s of packed weights over the rotation."""
+    out = []
+    for m, n, k in ((4096, 1024, 2), (42000, 1024, 2), (32768, 1024, 2), (42000, 1024, 3)):
+        wpr = amq.words_per_row(n)
+        bytes_one = m * k * wpr * 4 + m * k * 4 + m * 4
+        copies = max(2, min(400, -(-(300 << 20) // bytes_one)))
+        g = torch.Generator(device=dev)
+        g.manual_seed(6)
+        W = torch.randint(-2 ** 31, 2 ** 31 - 1, (copies, m, k, wpr), dtype=torch.int32, device=dev, generator=g)
+        Wa = torch.rand((copies, m, k), device=dev, generator=g) * 0.02
+        x = torch.rand((1, n), device=dev, generator=g) * 2 - 1
+        xc, xb = amq.quantize(x, k, 2)
+        y = torch.empty((copies, 1, m), device=dev)
+
+        def rotation():
+            for c in range(copies):
+                amq.binary_gemm(W[c], Wa[c], xc, xb, n, y=y[c])
+
+        line = {"workload": "batch-1 binary GEMV %d x %d, %d/%d bits, rotated over %d weight copies (%d MiB in all)" % (
+                    m, n, k, k, copies, copies * bytes_one >> 20), "bound": "hbm", "unit": "GB/s", "peak": peak,
+                "peak_kind": "of " + peak_kind, "algorithmic_bytes": int(copies * bytes_one)}
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                rotation()
+                with torch.cuda.graph(graph, stream=side):
+                    rotation()
+            torch.cuda.current_stream().wait_stream(side)
+            ms = _burst_ms(torch, graph.replay, 5)
+            line.update({"ms": ms, "us_per_launch": 1e3 * ms / copies, "achieved": copies * bytes_one / (ms * 1e-3) / 1e9})
+            line["frac"] = line["achieved"] / peak
+        except Exception as exc:
+            line["graph_replay_error"] = str(exc)[:120]
+        out.append(line)
+        del W, Wa, y
     return out
 
 
