@@ -34,8 +34,8 @@ amq_status enqueue_persistent(const CellCall& c, const CellWorkspace& ws, const 
                               const float* h0, const float* c0, float* h_seq, float* h_last, float* c_last,
                               cudaStream_t st)
 {
-    if (steps > 1)      // stale step tags must not match (a single step polls nothing)
-        AMQ_CUDA_TRY(cudaMemsetAsync(ws.hx, 0, (size_t)2 * c.H * 8, st));
+    // the caller has cleared the status words and, for more than one step, the exchange words behind them (stale
+    // step tags must not match; a single step polls nothing)
     return launch_rnn_persistent(c.Wcodes, c.Walpha, c.bias, c.I, c.H, c.k_w, c.k_a, c.T, c.gru, x_seq, steps,
                                  h0, c0, h_seq, h_last, c_last, ws.hx, ws.status, st);
 }
@@ -80,8 +80,9 @@ amq_status enqueue_sequence(const CellCall& c, const CellWorkspace& ws, const fl
                             cudaStream_t st)
 {
     const size_t state_bytes = (size_t)c.batch * c.H * sizeof(float);
-    AMQ_CUDA_TRY(cudaMemsetAsync(ws.status, 0, 256, st));
-    if (steps > 0 && use_persistent(c))
+    const bool persistent = steps > 0 && use_persistent(c);
+    AMQ_CUDA_TRY(cudaMemsetAsync(ws.status, 0, 256 + ((persistent && steps > 1) ? (size_t)2 * c.H * 8 : 0), st));
+    if (persistent)
         return enqueue_persistent(c, ws, x_seq, steps, h0, c0, h_seq, h_last, c_last, st);
     if (!c.gru) AMQ_CUDA_TRY(cudaMemcpyAsync(ws.c, c0, state_bytes, cudaMemcpyDeviceToDevice, st));
     const float* h_prev = h0;

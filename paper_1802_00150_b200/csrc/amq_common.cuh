@@ -54,12 +54,13 @@ inline CellWorkspace carve_cell_workspace(void* base, int I, int H, int batch, i
     char* p = static_cast<char*>(base);
     size_t off = 0;
     w.status = reinterpret_cast<uint32_t*>(p + off);            off += 256;
+    // the exchange words directly behind the status words: one memset clears both before a sequence
+    w.hx = reinterpret_cast<unsigned long long*>(p + off);      off += round_up((size_t)2 * H * 8, 256);
     w.zcodes = reinterpret_cast<uint32_t*>(p + off);            off += round_up((size_t)batch * k_a * words_per_row(I + H) * 4, 256);
     w.zbeta = reinterpret_cast<float*>(p + off);                off += round_up((size_t)batch * k_a * 4, 256);
     w.h[0] = reinterpret_cast<float*>(p + off);                 off += round_up((size_t)batch * H * 4, 256);
     w.h[1] = reinterpret_cast<float*>(p + off);                 off += round_up((size_t)batch * H * 4, 256);
     w.c = reinterpret_cast<float*>(p + off);                    off += round_up((size_t)batch * H * 4, 256);
-    w.hx = reinterpret_cast<unsigned long long*>(p + off);      off += round_up((size_t)2 * H * 8, 256);
     w.bytes = off;
     return w;
 }
