@@ -11,8 +11,9 @@
 // each and are subtracted again.  Expanding costs one shift (issued as a multiplication, on the FMA pipe)
 // and one three-input logic operation per four bytes: output register s of a 32-bit word keeps bits s,
 // s + 8, s + 16, s + 24 in its four bytes, i.e. the K positions inside a word are permuted, identically for
-// both operands, which a dot product does not see.  What bounds the expansion is the shared-memory store
-// bandwidth (128 operand bytes per row and stage), not the arithmetic.
+// both operands, which a dot product does not see.  What bounds the main loop is the shared-memory port, which
+// the expansion stores (128 operand bytes per row and stage) share with the operand reads of the MMAs
+// (an M 128 x N 256 x K 32 instruction reads 12 KB), not the arithmetic.
 //
 // Shared-memory operand layout: K-major with the 128-byte swizzle: a pipeline stage holds 128 bytes of K per
 // operand row, rows are 128 bytes apart, groups of 8 rows 1024 bytes apart, and the 16-byte chunk j of row r
@@ -28,6 +29,12 @@
 // completed.  A CTA may own two M tiles that share one expanded activation tile, which halves the
 // expansion work per MMA.  Every wait is bounded: when one runs out the CTA records the failure in a status
 // word, skips its stores, frees its tensor memory and returns.
+//
+// Two kernels share these pieces: bgemm_tc_kernel (one tile, or pair of M tiles, per CTA; all warps run the
+// epilogue after the last MMA) and bgemm_tc_persistent_kernel (one CTA per SM walks over tiles; accumulators
+// double-buffered in tensor memory, dedicated epilogue warps, so that the epilogue of a tile overlaps the main
+// loop of the next).  Both may be launched as programmatic dependents of the kernel that produces the
+// activation planes: they set themselves up and fetch weight rows, then wait for it.
 #include "amq_common.cuh"
 
 namespace amq {
@@ -155,15 +162,6 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld8(uint32_t taddr, int (&v)[8])
