@@ -414,6 +414,8 @@ def run_ours(args, wl):
             assert amq.device_status() == 0
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(wl, unit)
+            if not args.no_extras:
+                line["cpu_baseline_table6"] = cpu_baseline_table6()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
@@ -707,6 +709,32 @@ def greedy_decoding_line(amq, torch, dev):
                             V, H, ntok),
             "ms": ms, "bound": "latency", "us_per_token": 1e3 * ms / ntok, "tokens_per_s": ntok * 1e3 / ms,
             "distinct_tokens": int(torch.unique(tokens).numel())}
+
+
+def cpu_baseline_table6():
+    """The oracle, as it stands, on one host core, on the operations the paper times in Table 6 (on-line quantization of
+    the 1024-vector h plus the binary product; weights quantized beforehand, not timed): the same kind of measurement as
+    the paper's, on this machine's CPU and with a plain, untuned program."""
+    import oracle
+    out = []
+    h = synth.uniform((1, 1024), -1, 1, 11, 1).astype(np.float64)
+    for m, k in ((4096, 2), (4096, 3), (42000, 2), (42000, 3)):
+        rows = min(m, 4096)                                          # quantize a block of rows and tile it: only the product is timed
+        Wc, Wa = oracle.quantize_rows(synth.normal((rows, 1024), 0.05, 11, 2).astype(np.float64), k, 2)
+        reps = -(-m // rows)
+        Wc, Wa = np.tile(Wc, (reps, 1, 1))[:m], np.tile(Wa, (reps, 1))[:m]
+        best_q, best_p = 1e30, 1e30
+        for _ in range(3):
+            t0 = time.perf_counter()
+            hc, hb = oracle.quantize_rows(h, k, 2)
+            t1 = time.perf_counter()
+            oracle.binary_gemm(Wc, Wa, hc, hb, 1024)
+            t2 = time.perf_counter()
+            best_q, best_p = min(best_q, t1 - t0), min(best_p, t2 - t1)
+        out.append({"workload": "Table 6 shape %d x 1024, %d/%d bits, batch 1: oracle on one host core" % (m, k, k),
+                    "quantize_ms": 1e3 * best_q, "product_ms": 1e3 * best_p, "total_ms": 1e3 * (best_q + best_p),
+                    "cores": 1, "kind": "oracle", "sample": "best of 3; weights quantized beforehand"})
+    return out
 
 
 def cpu_baseline(wl, unit):
