@@ -87,3 +87,62 @@ def test_argument_validation_happens_on_the_host(lib):
     assert s(fake, fake, None, 8, 8, 2, fake, fake, fake, 1, 2, 2, fake, fake, fake, 16, None) == -4   # workspace small
     assert s(fake, fake, None, 8, 8, 2, fake, fake, fake, 1, 2, 2, fake, fake, None, 1 << 20, None) == -4
     assert s(fake, fake, None, 8, 8, 2, fake, fake, fake, 1, 2, 2, fake, fake, fake, 1 << 20, None) == -1  # h_out == h_in
+
+
+def test_argument_validation_of_the_widened_entry_points(lib):
+    """Variants of the quantizer, the paper-form cell, the original-form GRU, the output layer and the decoding loop:
+    every rejection below is decided on the host, before any launch (the pointers are never dereferenced)."""
+    vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    fake, fake2, odd = vp(0x1000), vp(0x2000), vp(0x1004)
+    qv = lib.amq_quantize_variant
+    qv.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp]
+    assert qv(fake, 1, 8, 8, 2, 2, 2, 0, fake, fake, None) == -2           # unknown method
+    assert qv(fake, 1, 8, 8, 2, 2, -1, 0, fake, fake, None) == -2
+    assert qv(fake, 1, 8, 8, 5, 2, 1, 0, fake, fake, None) == -2           # k
+    assert qv(fake, 1, 8, 4, 2, 2, 1, 1, fake, fake, None) == -1           # ldx < n
+    assert qv(fake, 1, 8, 8, 2, 2, 1, 1, odd, fake, None) == -3
+    assert qv(None, 0, 8, 8, 2, 2, 1, 1, None, None, None) == 0            # empty input
+    sm = lib.amq_log_softmax_argmax
+    sm.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp]
+    assert sm(fake, 1, 0, 0, fake, 0, fake, None) == -1                    # n < 1
+    assert sm(fake, 1, 8, 4, fake, 8, fake, None) == -1                    # ld < n
+    assert sm(fake, 1, 8, 8, fake, 4, fake, None) == -1                    # ldp < n
+    assert sm(fake, 1, 8, 8, None, 8, None, None) == -1                    # nothing to write
+    assert sm(None, 0, 8, 8, None, 8, None, None) == 0
+    er = lib.amq_embedding_rows
+    er.argtypes = [vp, vp, ci, ci, ci, vp, ci, vp, vp, vp]
+    assert er(fake, fake, 10, 8, 5, fake, 1, fake, fake, None) < 0         # k
+    assert er(fake, fake, 0, 8, 2, fake, 1, fake, fake, None) < 0          # empty vocabulary
+    lib.amq_gru_original_workspace_bytes.restype = sz
+    lib.amq_gru_original_workspace_bytes.argtypes = [ci, ci, ci, ci]
+    need = lib.amq_gru_original_workspace_bytes(8, 8, 2, 2)
+    assert need > 0 and lib.amq_gru_original_workspace_bytes(8, 8, 2, 5) == 0 and lib.amq_gru_original_workspace_bytes(8, 0, 2, 2) == 0
+    go = lib.amq_gru_step_original
+    go.argtypes = [vp, vp, vp, ci, ci, ci, vp, vp, ci, ci, ci, vp, vp, sz, vp]
+    assert go(fake, fake, None, 8, 8, 2, fake, fake, 2, 2, 2, fake2, fake, need - 1, None) == -4
+    assert go(fake, fake, None, 8, 8, 2, fake, fake, 2, 2, 2, fake, fake, need, None) == -1       # h_out == h_in
+    assert go(fake, fake, None, 8, 8, 0, fake, fake, 2, 2, 2, fake2, fake, need, None) == -2      # k_w
+    assert go(odd, fake, None, 8, 8, 2, fake, fake, 2, 2, 2, fake2, fake, need, None) == -3
+    assert go(fake, fake, None, 8, 8, 2, fake, fake, 0, 2, 2, fake2, fake, need, None) == 0       # empty batch
+    lib.amq_lm_decode_workspace_bytes.restype = sz
+    lib.amq_lm_decode_workspace_bytes.argtypes = [ci] * 5
+    dneed = lib.amq_lm_decode_workspace_bytes(100, 8, 8, 2, 2)
+    assert dneed >= 100 * 4 and lib.amq_lm_decode_workspace_bytes(0, 8, 8, 2, 2) == 0
+    dec = lib.amq_lm_greedy_decode
+    dec.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, vp, ci, ci, vp, vp, vp, ci, ci, ci, vp, ci, vp, vp, vp, vp, sz, vp]
+    args = [fake, fake, 100, 8, 2, fake, fake, fake, fake, None, 8, 2, fake, fake, None, 2, 2, 2, fake, 3, fake, fake, None,
+            fake, dneed, None]
+    bad = list(args); bad[24] = dneed - 1
+    assert dec(*bad) == -4                                                 # workspace too small
+    bad = list(args); bad[15] = 7
+    assert dec(*bad) == -2                                                 # bits of the output layer
+    bad = list(args); bad[12] = None
+    assert dec(*bad) == -1                                                 # no output matrix
+    bad = list(args); bad[0] = odd
+    assert dec(*bad) == -3
+    bad = list(args); bad[19] = 0
+    assert dec(*bad) == 0                                                  # no steps: nothing to do
+    lib.amq_lstm_paper_workspace_bytes.restype = sz
+    lib.amq_lstm_paper_workspace_bytes.argtypes = [ci] * 4
+    assert lib.amq_lstm_paper_workspace_bytes(8, 2, 3, 2) > lib.amq_lstm_paper_workspace_bytes(8, 2, 1, 2) > 0
+    assert lib.amq_lstm_paper_workspace_bytes(8, 2, 3, 0) == 0
