@@ -27,6 +27,7 @@ struct GemvParams {
     int32_t* D;                 // EPI_DOTS: [m][k_w][k_a]
     int m, n, CH;
     int epilogue;
+    bool overlap;               // host side only: launch as a programmatic dependent of the preceding kernel
 };
 
 // differing bits of (w xor x) over the four words of a chunk, accumulated carry-save:
@@ -64,6 +65,7 @@ template <int KW, int KA, int CPT, int R, int SEG_LOG2, bool EXACT>
 __global__ void __launch_bounds__(256)
 bgemv_kernel(GemvParams p)
 {
+    grid_dependency_wait();     // the activation planes may come from the preceding kernel of the stream
     const int lane = threadIdx.x & 31;
     constexpr int SEG = 1 << SEG_LOG2;
     constexpr int spw = 32 >> SEG_LOG2;            // rows per load instruction of the warp
@@ -81,11 +83,11 @@ bgemv_kernel(GemvParams p)
         has[c] = EXACT || (sub + c * SEG < CH);
 #pragma unroll
         for (int j = 0; j < KA; ++j)
-            xr[j][c] = has[c] ? __ldg(p.x + (size_t)j * CH + sub + c * SEG) : make_uint4(0, 0, 0, 0);
+            xr[j][c] = has[c] ? p.x[(size_t)j * CH + sub + c * SEG] : make_uint4(0, 0, 0, 0);   // ordinary load, L1-cached
     }
     float beta[KA];
 #pragma unroll
-    for (int j = 0; j < KA; ++j) beta[j] = (p.epilogue == EPI_Y) ? __ldg(p.xbeta + j) : 0.0f;
+    for (int j = 0; j < KA; ++j) beta[j] = (p.epilogue == EPI_Y) ? p.xbeta[j] : 0.0f;
 
     const long long blocks = ((long long)p.m + 31) >> 5;
     const long long warp_global = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -208,7 +210,7 @@ amq_status launch_cfg(const GemvParams& p, cudaStream_t st)
     const long long need = (passes + 7) / 8;                            // small matrices: one pass per warp, spread over the SMs
     const int limit = cached_grid[exact ? 1 : 0];
     const int grid = (int)(need < limit ? need : limit);
-    kernel<<<grid, 256, 0, st>>>(p);
+    AMQ_CUDA_TRY(launch_kernel(kernel, dim3((unsigned)grid), dim3(256), 0, st, p.overlap, p));
     AMQ_LAUNCH_CHECK();
     return AMQ_OK;
 }
@@ -256,6 +258,7 @@ amq_status launch_binary_gemv(const GemmArgs& a, cudaStream_t st)
     p.D = a.D;
     p.m = a.m; p.n = a.n; p.CH = words_per_row(a.n) / 4;
     p.epilogue = a.epilogue;
+    p.overlap = a.overlap_with_previous;
     switch (a.k_w) {
         case 1: return launch_ka<1>(p, a.k_a, st);
         case 2: return launch_ka<2>(p, a.k_a, st);

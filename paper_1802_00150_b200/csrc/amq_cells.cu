@@ -40,16 +40,17 @@ amq_status enqueue_persistent(const CellCall& c, const CellWorkspace& ws, const 
                                  h0, c0, h_seq, h_last, c_last, ws.hx, ws.status, st);
 }
 
-__global__ void lstm_gates_kernel(const float* __restrict__ pre, const float* __restrict__ addend, const float* __restrict__ c_in,
-                                  float* __restrict__ h_out, float* __restrict__ c_out, int H)
+// (inputs come from the preceding kernels of the stream: ordinary loads after the wait, no read-only path)
+__global__ void lstm_gates_kernel(const float* pre, const float* addend, const float* c_in, float* h_out, float* c_out, int H)
 {
+    grid_dependency_wait();
     const int u = blockIdx.x * blockDim.x + threadIdx.x;
     if (u >= H) return;
     float g4[4];
 #pragma unroll
-    for (int g = 0; g < 4; ++g) g4[g] = pre[g * H + u] + (addend ? addend[g * H + u] : 0.0f);
+    for (int g = 0; g < 4; ++g) g4[g] = __ldcg(pre + g * H + u) + (addend ? __ldcg(addend + g * H + u) : 0.0f);
     const float ig = 1.0f / (1.0f + __expf(-g4[0])), fg = 1.0f / (1.0f + __expf(-g4[1])), og = 1.0f / (1.0f + __expf(-g4[2]));
-    const float c = fg * c_in[u] + ig * tanhf(g4[3]);
+    const float c = fg * __ldcg(c_in + u) + ig * tanhf(g4[3]);
     c_out[u] = c;
     h_out[u] = og * tanhf(c);
 }
@@ -167,9 +168,10 @@ amq_status sequence_host_entry(const CellCall& c, const float* x_seq_host, int s
 }  // namespace
 
 amq_status launch_lstm_gates(const float* pre, const float* addend, const float* c_in, float* h_out, float* c_out, int H,
-                             cudaStream_t st)
+                             cudaStream_t st, bool overlap_with_previous)
 {
-    lstm_gates_kernel<<<(unsigned)((H + 255) / 256), 256, 0, st>>>(pre, addend, c_in, h_out, c_out, H);
+    AMQ_CUDA_TRY(launch_kernel(lstm_gates_kernel, dim3((unsigned)((H + 255) / 256)), dim3(256), 0, st, overlap_with_previous,
+                               pre, addend, c_in, h_out, c_out, H));
     AMQ_LAUNCH_CHECK();
     return AMQ_OK;
 }

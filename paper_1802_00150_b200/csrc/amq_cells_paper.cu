@@ -78,16 +78,18 @@ amq_status recurrent_part(const PaperCall& c, const PaperWorkspace& ws, const fl
     a.epilogue = EPI_LSTM; a.H = c.H;
     // in a sequence the kernel before this quantizer is the recurrent product of the previous timestep: when that
     // runs as a single wave the quantizer may be scheduled behind it early (it waits for it first thing)
+    // (with one sequence every kernel of the step is short and waits for its predecessor first thing: all overlapped)
     amq_status s = launch_quantize(h_in, c.H, c.H, nullptr, 0, 0, c.batch, c.k_a, c.T, ws.hcodes, ws.hbeta, st,
-                                   gemm_tc_single_wave(a));
+                                   c.batch == 1 || gemm_tc_single_wave(a));
     if (s != AMQ_OK) return s;
     if (c.batch == 1) {
         // one sequence: the bandwidth-bound matrix-vector kernel writes the pre-activations, a small kernel applies the gates
         a.epilogue = EPI_Y; a.y = ws.gates; a.ldy = 4 * c.H;
         if (gemv_supported(a)) {
+            a.overlap_with_previous = true;
             s = launch_binary_gemv(a, st);
             if (s != AMQ_OK) return s;
-            return launch_lstm_gates(ws.gates, proj, c_in, h_out, c_out, c.H, st);
+            return launch_lstm_gates(ws.gates, proj, c_in, h_out, c_out, c.H, st, true);
         }
     }
     a.y = nullptr; a.ldy = 0;

@@ -100,6 +100,22 @@ struct GemmArgs {
 // earlier than its exit: measured, early signals only made the waiting CTAs take SM resources sooner.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Launch `kernel`, as a programmatic dependent of the preceding kernel of the stream when `overlap` is set (the kernel
+// must then execute grid_dependency_wait() before it reads or writes anything another kernel of the chain touches,
+// and read such data with ordinary loads, not through the read-only path).
+template <typename... Params, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool overlap,
+                                 Args... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr; cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 amq_status launch_binary_gemm(const GemmArgs& a, cudaStream_t st);
 // whether the tensor-core kernel takes the problem with all its CTAs resident at once (then the quantizer of the next
 // timestep is launched as its programmatic dependent: its CTAs move in as the product's CTAs exit)
@@ -108,7 +124,12 @@ bool gemm_tc_single_wave(const GemmArgs& a);
 // Batch-1 streaming kernel (EPI_DOTS / EPI_Y): whether it covers a problem, and its launch.
 // gates of Eq. 6 for one sequence from pre-activations pre[4H] (+ addend[4H] when given), rows i, f, o, g
 amq_status launch_lstm_gates(const float* pre, const float* addend, const float* c_in, float* h_out, float* c_out, int H,
-                             cudaStream_t st);
+                             cudaStream_t st, bool overlap_with_previous = false);
+// gather of rows of a quantized embedding / log-softmax and arg-max of rows of logits (validated arguments)
+amq_status launch_embedding_rows(const uint32_t* We_codes, const float* We_alpha, int vocab, int n, int k, const int32_t* tokens,
+                                 int count, uint32_t* xcodes, float* xbeta, cudaStream_t st, bool overlap_with_previous);
+amq_status launch_log_softmax_argmax(const float* logits, int rows, int n, int ld, float* logp, int ldp, int32_t* argmax,
+                                     cudaStream_t st, bool overlap_with_previous);
 bool gemv_supported(const GemmArgs& a);
 amq_status launch_binary_gemv(const GemmArgs& a, cudaStream_t st);
 

@@ -67,22 +67,33 @@ amq_status amq_lm_greedy_decode(const uint32_t* We_codes, const float* We_alpha,
     if (!tokens || !h || !c) return AMQ_ERR_INVALID_ARG;
     const amq::DecodeWorkspace ws = amq::carve(workspace, vocab, I, H, k_e, k_a);
     cudaStream_t st = (cudaStream_t)stream;
-    amq_status s = amq_quantize(h, 1, H, H, k_a, T, ws.hcodes, ws.hbeta, stream);          // h_hat of the start state
+    // every launch after the first is a programmatic dependent of its predecessor (each kernel waits for it first
+    // thing), which takes most of the gaps between these short kernels out of the chain
+    auto product = [&](const uint32_t* Wc, const float* Wa, int m, int n, int kw, const uint32_t* xc, const float* xb, int ka,
+                       const float* b, float* y) {
+        amq::GemmArgs a{};
+        a.Wcodes = Wc; a.Walpha = Wa; a.m = m; a.n = n; a.k_w = kw;
+        a.xcodes = xc; a.xbeta = xb; a.batch = 1; a.k_a = ka;
+        a.bias = b; a.epilogue = amq::EPI_Y; a.y = y; a.ldy = m;
+        a.overlap_with_previous = true;
+        return amq::launch_binary_gemm(a, st);
+    };
+    amq_status s = amq::launch_quantize(h, H, H, nullptr, 0, 0, 1, k_a, T, ws.hcodes, ws.hbeta, st, false);   // h_hat of the start state
     for (int t = 0; t < steps && s == AMQ_OK; ++t) {
-        s = amq_embedding_rows(We_codes, We_alpha, vocab, I, k_e, tokens + t, 1, ws.xcodes, ws.xbeta, stream);
+        s = amq::launch_embedding_rows(We_codes, We_alpha, vocab, I, k_e, tokens + t, 1, ws.xcodes, ws.xbeta, st, true);
         if (s != AMQ_OK) break;
-        s = amq_binary_gemm(Wi_codes, Wi_alpha, 4 * H, I, k_w, ws.xcodes, ws.xbeta, 1, k_e, bias, ws.proj, 4 * H, stream);
+        s = product(Wi_codes, Wi_alpha, 4 * H, I, k_w, ws.xcodes, ws.xbeta, k_e, bias, ws.proj);
         if (s != AMQ_OK) break;
-        s = amq_binary_gemm(Wh_codes, Wh_alpha, 4 * H, H, k_w, ws.hcodes, ws.hbeta, 1, k_a, nullptr, ws.pre, 4 * H, stream);
+        s = product(Wh_codes, Wh_alpha, 4 * H, H, k_w, ws.hcodes, ws.hbeta, k_a, nullptr, ws.pre);
         if (s != AMQ_OK) break;
-        s = amq::launch_lstm_gates(ws.pre, ws.proj, c, h, c, H, st);                        // state updated in place
+        s = amq::launch_lstm_gates(ws.pre, ws.proj, c, h, c, H, st, true);                  // state updated in place
         if (s != AMQ_OK) break;
-        s = amq_quantize(h, 1, H, H, k_a, T, ws.hcodes, ws.hbeta, stream);
+        s = amq::launch_quantize(h, H, H, nullptr, 0, 0, 1, k_a, T, ws.hcodes, ws.hbeta, st, true);
         if (s != AMQ_OK) break;
-        s = amq_binary_gemm(Ws_codes, Ws_alpha, vocab, H, k_s, ws.hcodes, ws.hbeta, 1, k_a, bias_s, ws.logits, vocab, stream);
+        s = product(Ws_codes, Ws_alpha, vocab, H, k_s, ws.hcodes, ws.hbeta, k_a, bias_s, ws.logits);
         if (s != AMQ_OK) break;
-        s = amq_log_softmax_argmax(ws.logits, 1, vocab, vocab, logp ? logp + (size_t)t * vocab : nullptr, vocab, tokens + t + 1,
-                                   stream);
+        s = amq::launch_log_softmax_argmax(ws.logits, 1, vocab, vocab, logp ? logp + (size_t)t * vocab : nullptr, vocab,
+                                           tokens + t + 1, st, true);
     }
     return s;
 }

@@ -43,20 +43,36 @@ __global__ void unpack_kernel(const uint32_t* __restrict__ codes, const float* _
 // One thread per 128-bit chunk of the gathered rows: out row c <- table row tokens[c] (codes), and the row's
 // coefficients by the first k threads of the row.
 __global__ void embedding_rows_kernel(const uint4* __restrict__ codes, const float* __restrict__ coeffs, int vocab,
-                                      const int32_t* __restrict__ tokens, size_t count, int k, int chunks /* k * wpr / 4 */,
+                                      const int32_t* tokens, size_t count, int k, int chunks /* k * wpr / 4 */,
                                       uint4* __restrict__ out_codes, float* __restrict__ out_coeffs)
 {
+    grid_dependency_wait();             // the token ids may come from the preceding kernel (greedy decoding)
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= count * (size_t)chunks) return;
     const size_t row = idx / chunks;
     const int c = (int)(idx - row * chunks);
-    int tok = __ldg(tokens + row);
+    int tok = __ldcg(tokens + row);
     tok = tok < 0 ? 0 : (tok >= vocab ? vocab - 1 : tok);          // out-of-range ids are clamped, never dereferenced
     out_codes[idx] = __ldg(codes + (size_t)tok * chunks + c);
     if (c < k) out_coeffs[row * k + c] = __ldg(coeffs + (size_t)tok * k + c);
 }
 
 }  // namespace
+
+amq_status launch_embedding_rows(const uint32_t* We_codes, const float* We_alpha, int vocab, int n, int k, const int32_t* tokens,
+                                 int count, uint32_t* xcodes, float* xbeta, cudaStream_t st, bool overlap_with_previous)
+{
+    const int chunks = k * words_per_row(n) / 4;
+    const size_t total = (size_t)count * chunks;
+    const size_t blocks = (total + 255) / 256;
+    if (blocks > 0x7fffffffull) return AMQ_ERR_UNSUPPORTED;
+    AMQ_CUDA_TRY(launch_kernel(embedding_rows_kernel, dim3((unsigned)blocks), dim3(256), 0, st, overlap_with_previous,
+                               reinterpret_cast<const uint4*>(We_codes), We_alpha, vocab, tokens, (size_t)count, k, chunks,
+                               reinterpret_cast<uint4*>(xcodes), xbeta));
+    AMQ_LAUNCH_CHECK();
+    return AMQ_OK;
+}
+
 }  // namespace amq
 
 extern "C" {
@@ -110,15 +126,7 @@ amq_status amq_embedding_rows(const uint32_t* We_codes, const float* We_alpha, i
     if (count == 0) return AMQ_OK;
     if (!We_codes || !We_alpha || !tokens || !xcodes || !xbeta) return AMQ_ERR_INVALID_ARG;
     if (!amq::aligned16(We_codes) || !amq::aligned16(xcodes)) return AMQ_ERR_ALIGNMENT;
-    const int chunks = k * amq::words_per_row(n) / 4;
-    const size_t total = (size_t)count * chunks;
-    const size_t blocks = (total + 255) / 256;
-    if (blocks > 0x7fffffffull) return AMQ_ERR_UNSUPPORTED;
-    amq::embedding_rows_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(
-        reinterpret_cast<const uint4*>(We_codes), We_alpha, vocab, tokens, (size_t)count, k, chunks,
-        reinterpret_cast<uint4*>(xcodes), xbeta);
-    AMQ_LAUNCH_CHECK();
-    return AMQ_OK;
+    return amq::launch_embedding_rows(We_codes, We_alpha, vocab, n, k, tokens, count, xcodes, xbeta, (cudaStream_t)stream, false);
 }
 
 amq_status amq_unpack(const uint32_t* codes, const float* coeffs, int rows, int n, int k,

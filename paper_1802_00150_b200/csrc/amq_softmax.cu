@@ -48,9 +48,10 @@ __device__ __forceinline__ float block_sum(float sum, float* s_sum)
 constexpr int VEC = 12;
 
 __global__ void __launch_bounds__(SM_THREADS)
-log_softmax_argmax_resident_kernel(const float* __restrict__ logits, int n, int ld, float* __restrict__ logp, int ldp,
+log_softmax_argmax_resident_kernel(const float* logits, int n, int ld, float* __restrict__ logp, int ldp,
                                    int32_t* __restrict__ arg)
 {
+    grid_dependency_wait();             // the logits come from the preceding kernel of the stream
     __shared__ float s_val[32];
     __shared__ int s_idx[32];
     __shared__ float s_sum[32];
@@ -61,10 +62,10 @@ log_softmax_argmax_resident_kernel(const float* __restrict__ logits, int n, int 
 #pragma unroll
     for (int q = 0; q < VEC; ++q) {
         const int t4 = tid + q * SM_THREADS;
-        v[q] = t4 < n4 ? __ldg(reinterpret_cast<const float4*>(z) + t4) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        v[q] = t4 < n4 ? __ldcg(reinterpret_cast<const float4*>(z) + t4) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
     }
     const int tail = n4 * 4 + tid;                                  // at most three tail elements, one per thread
-    const float vt = tail < n ? __ldg(z + tail) : -INFINITY;
+    const float vt = tail < n ? __ldcg(z + tail) : -INFINITY;
 
     float mv = vt;
     int mi = tail < n ? tail : 0x7fffffff;
@@ -104,9 +105,10 @@ log_softmax_argmax_resident_kernel(const float* __restrict__ logits, int n, int 
 }
 
 __global__ void __launch_bounds__(SM_THREADS)
-log_softmax_argmax_kernel(const float* __restrict__ logits, int n, int ld, float* __restrict__ logp, int ldp,
+log_softmax_argmax_kernel(const float* logits, int n, int ld, float* __restrict__ logp, int ldp,
                           int32_t* __restrict__ arg)
 {
+    grid_dependency_wait();             // the logits come from the preceding kernel of the stream
     __shared__ float s_val[32];
     __shared__ int s_idx[32];
     __shared__ float s_sum[32];
@@ -116,7 +118,7 @@ log_softmax_argmax_kernel(const float* __restrict__ logits, int n, int ld, float
     // pass 1: maximum and its first index
     float mv = -INFINITY;
     int mi = 0x7fffffff;
-    for (int t = tid; t < n; t += SM_THREADS) max_combine(mv, mi, __ldg(z + t), t);
+    for (int t = tid; t < n; t += SM_THREADS) max_combine(mv, mi, __ldcg(z + t), t);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1)
         max_combine(mv, mi, __shfl_xor_sync(0xffffffffu, mv, off), __shfl_xor_sync(0xffffffffu, mi, off));
@@ -129,7 +131,7 @@ log_softmax_argmax_kernel(const float* __restrict__ logits, int n, int ld, float
 
     // pass 2: sum of exp(z - max), fixed order (thread-strided, then butterflies)
     float sum = 0.0f;
-    for (int t = tid; t < n; t += SM_THREADS) sum += __expf(__ldg(z + t) - mv);
+    for (int t = tid; t < n; t += SM_THREADS) sum += __expf(__ldcg(z + t) - mv);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
     if (lane == 0) s_sum[warp] = sum;
@@ -141,12 +143,23 @@ log_softmax_argmax_kernel(const float* __restrict__ logits, int n, int ld, float
 
     if (logp) {
         float* out = logp + (size_t)blockIdx.x * ldp;
-        for (int t = tid; t < n; t += SM_THREADS) out[t] = __ldg(z + t) - lse;
+        for (int t = tid; t < n; t += SM_THREADS) out[t] = __ldcg(z + t) - lse;
     }
     if (arg && tid == 0) arg[blockIdx.x] = mi;
 }
 
 }  // namespace
+
+amq_status launch_log_softmax_argmax(const float* logits, int rows, int n, int ld, float* logp, int ldp, int32_t* argmax,
+                                     cudaStream_t st, bool overlap_with_previous)
+{
+    const bool resident = n <= SM_THREADS * 4 * VEC && (ld & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;
+    AMQ_CUDA_TRY(launch_kernel(resident ? log_softmax_argmax_resident_kernel : log_softmax_argmax_kernel, dim3((unsigned)rows),
+                               dim3(SM_THREADS), 0, st, overlap_with_previous, logits, n, ld, logp, ldp, argmax));
+    AMQ_LAUNCH_CHECK();
+    return AMQ_OK;
+}
+
 }  // namespace amq
 
 extern "C" amq_status amq_log_softmax_argmax(const float* logits, int rows, int n, int ld,
@@ -155,11 +168,5 @@ extern "C" amq_status amq_log_softmax_argmax(const float* logits, int rows, int 
     if (rows < 0 || n < 1 || ld < n || (logp && ldp < n)) return AMQ_ERR_INVALID_ARG;
     if (rows == 0) return AMQ_OK;
     if (!logits || (!logp && !argmax)) return AMQ_ERR_INVALID_ARG;
-    const bool resident = n <= amq::SM_THREADS * 4 * amq::VEC && (ld & 3) == 0 && (reinterpret_cast<uintptr_t>(logits) & 15) == 0;
-    if (resident)
-        amq::log_softmax_argmax_resident_kernel<<<(unsigned)rows, amq::SM_THREADS, 0, (cudaStream_t)stream>>>(logits, n, ld, logp, ldp, argmax);
-    else
-        amq::log_softmax_argmax_kernel<<<(unsigned)rows, amq::SM_THREADS, 0, (cudaStream_t)stream>>>(logits, n, ld, logp, ldp, argmax);
-    AMQ_LAUNCH_CHECK();
-    return AMQ_OK;
+    return amq::launch_log_softmax_argmax(logits, rows, n, ld, logp, ldp, argmax, (cudaStream_t)stream, false);
 }

@@ -184,3 +184,26 @@ def test_native_greedy_decoding_equals_the_composed_calls_and_the_oracle_on_its_
     lp_o, _ = oracle.log_softmax_argmax(z_o)
     tol = parity.output_tolerance(Wsa, hb_o, H).max()
     assert np.abs(logp[0].cpu().numpy() - lp_o[0]).max() <= 2 * tol + 2e-5
+
+
+def test_native_greedy_decoding_repeats_bit_for_bit(amq):
+    """The kernels of the decoding chain are launched as programmatic dependents of one another (each waits for its
+    predecessor first thing): a read that slipped ahead of a wait would show as run-to-run differences."""
+    I, H, V, k, steps = 128, 256, 5000, 2, 24
+    g = torch.Generator(device="cuda")
+    g.manual_seed(7)
+    q = lambda shape, std: amq.quantize(torch.randn(shape, device="cuda", generator=g) * std, k, 2)
+    (Wic, Wia), (Whc, Wha), (Wec, Wea), (Wsc, Wsa) = q((4 * H, I), 0.05), q((4 * H, H), 0.05), q((V, I), 0.5), q((V, H), 0.08)
+    bs = torch.randn((V,), device="cuda", generator=g) * 0.1
+    ws = amq.new_decode_workspace(V, I, H, k, k)
+    runs = []
+    for _ in range(5):
+        tokens = torch.zeros((steps + 1,), dtype=torch.int32, device="cuda")
+        tokens[0] = 3
+        h, c = torch.zeros((1, H), device="cuda"), torch.zeros((1, H), device="cuda")
+        logp = torch.empty((steps, V), device="cuda")
+        amq.lm_greedy_decode(Wec, Wea, Wic, Wia, Whc, Wha, None, Wsc, Wsa, bs, I, H, k, 2, tokens, h, c, ws, logp=logp)
+        runs.append((tokens.clone(), h.clone(), c.clone(), logp.clone()))
+    for r in runs[1:]:
+        assert all(torch.equal(a, b) for a, b in zip(r, runs[0]))
+    assert torch.unique(runs[0][0]).numel() > 3
