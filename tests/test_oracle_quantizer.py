@@ -360,3 +360,27 @@ def test_variants_final_refit_and_refined_greedy():
         a, b = oracle.quantize_variant(x[r], 3, 2, oracle.METHOD_ALTERNATING, True)
         assert np.array_equal(coeffs[r], a)
         assert np.array_equal(codes[r], oracle.pack_planes(b))
+
+
+def test_error_levels_of_the_methods_are_those_of_table_1_on_gaussian_rows():
+    """Table 1 prints the relative MSE of greedy, refined and alternating quantization of trained LSTM weights.  Those
+    weights are not available; rows of Gaussian noise are close to them in shape, and the oracle must then land near the
+    printed numbers: alternating (T = 2) within 15 %, the two baselines within 30 %, and in the printed order."""
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "table1_relative_mse.txt")
+    table = {}
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        parts = line.split()
+        table[parts[0]] = [float(v) for v in parts[1:]]
+    rows = synth.normal((48, 1024), 1.0, 77, 1).astype(np.float64)
+    norm = (rows ** 2).sum()
+    for col, k in enumerate((2, 3, 4)):
+        err = {}
+        for name, fn in (("greedy", lambda w: oracle.greedy(w, k)), ("refined", lambda w: oracle.refined_greedy(w, k)),
+                         ("alternating", lambda w: oracle.quantize(w, k, 2))):
+            err[name] = sum(oracle.objective(w, *fn(w)) for w in rows) / norm
+        assert err["greedy"] > err["refined"] > err["alternating"]
+        assert abs(err["alternating"] / table["alternating"][col] - 1) < 0.15, (k, err)
+        assert abs(err["greedy"] / table["greedy"][col] - 1) < 0.30, (k, err)
+        assert abs(err["refined"] / table["refined"][col] - 1) < 0.30, (k, err)
