@@ -821,8 +821,8 @@ int sm_count()
     return count;
 }
 
-// The persistent form: one M tile per CTA step, two accumulator buffers, dedicated epilogue warps.  Possible when
-// both buffers fit tensor memory and there are more tiles than SMs (otherwise nothing could overlap).
+// The persistent form: one M tile per CTA step, dedicated epilogue warps, two accumulator buffers when they fit tensor
+// memory.  Possible when there are more tiles than SMs (otherwise nothing could overlap).
 bool plan_persistent(const TcParams& base, int mtiles, int btiles, TcPlan* out)
 {
     TcParams p = base;
@@ -833,10 +833,13 @@ bool plan_persistent(const TcParams& base, int mtiles, int btiles, TcPlan* out)
     p.ntiles = mtiles * btiles;
     if (p.ntiles <= sms) return false;
     const int acc_cols = p.nseg * p.n_mma;
-    if (2 * acc_cols > 512) return false;
-    p.nbuf = 2;
+    if (acc_cols > 512) return false;
+    // two accumulator buffers when they fit (the epilogue of a tile then overlaps the MMAs of the next); with one (the
+    // GRU's two column segments at N = 192) the MMAs of the next tile wait for the epilogue, but its stages are expanded
+    // meanwhile and the CTA pays its set-up once: still ahead of three waves of the plain form (measured)
+    p.nbuf = (2 * acc_cols > 512) ? 1 : 2;
     int cols = 32;
-    while (cols < 2 * acc_cols) cols <<= 1;
+    while (cols < p.nbuf * acc_cols) cols <<= 1;
     p.tmem_cols = cols;
     const size_t stage = (size_t)128 * (TILE_M + p.n_mma);
     p.yt_bytes = (int)(((size_t)p.nseg * TILE_M * (p.TB + 1) * 4 + 15) / 16 * 16);

@@ -222,6 +222,7 @@ CELL_CASES = [
     ("gru", 33, 31, 1, 4, 2),
     ("lstm", 40, 640, 4, 4, 70),          # 160 tiles: gate epilogues of the persistent tensor-core kernel
     ("gru", 64, 800, 4, 1, 200),
+    ("gru", 32, 1500, 4, 4, 40),          # 150 tiles, two column segments of N = 192: persistent kernel, one accumulator buffer
     # batch 1 goes through the persistent weight-stationary kernel
     ("lstm", 1024, 1024, 2, 2, 1),        # the hidden-1024 layer of the benchmark, one step
     ("lstm", 1536, 1024, 3, 3, 1),        # n = 2560: sixteen elements per thread
