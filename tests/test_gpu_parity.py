@@ -420,7 +420,9 @@ def test_gru_step_in_the_original_form_matches_oracle(amq, I, H, kw, ka, batch):
     assert amq.device_status() == 0
 
 
-@pytest.mark.parametrize("cell,I,H,kw,ka,batch,steps", [("lstm", 256, 256, 2, 2, 20, 6), ("gru", 256, 192, 2, 3, 33, 5)])
+@pytest.mark.parametrize("cell,I,H,kw,ka,batch,steps", [("lstm", 256, 256, 2, 2, 20, 6), ("gru", 256, 192, 2, 3, 33, 5),
+                                                        ("gru", 32, 1500, 4, 4, 40, 4),      # persistent kernel, one buffer
+                                                        ("lstm", 64, 1280, 4, 4, 70, 4)])    # persistent kernel, two buffers
 def test_batched_sequences_repeat_bit_for_bit(amq, cell, I, H, kw, ka, batch, steps):
     """The product kernel of a timestep is launched so that it may start while the quantizer of that timestep still
     runs (it waits for it before reading the planes).  A read that slipped ahead of that wait would show up as results
