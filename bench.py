@@ -559,6 +559,7 @@ def batched_lines(amq, torch, dev, flush, hbm_peak, peak_kind):
                         "peak_kind": "of " + peak_kind, "algorithmic_bytes": int(alg)})
         del W, Wcodes, Walpha, acts, xc, xb, y
     out.append(paper_form_line(amq, torch, dev))
+    out.append(gru_forms_line(amq, torch, dev))
     out.append(greedy_decoding_line(amq, torch, dev))
     out.extend(table6_lines(amq, torch, dev, flush))
     out.append(quality_line(amq, torch, dev))
@@ -592,6 +593,25 @@ def paper_form_line(amq, torch, dev):
                         "one batched input projection + per-step quantize(h) and W_h product)" % (batch, steps),
             "ms": ms, "bound": "tensor+latency", "us_per_timestep": 1e3 * ms / steps,
             "timesteps_per_s": batch * steps / (ms * 1e-3)}
+
+
+def gru_forms_line(amq, torch, dev):
+    """One GRU timestep at the C4 shape (I = H = 2048, 2/3 bits, 256 sequences) in the two forms: the default one (reset
+    gate after the product: one quantization, one product) and the original one of Cho et al. (reset gate before the
+    candidate's product: two quantizations, two products)."""
+    wl = synth.WORKLOADS["gru2048_b256"]
+    g = torch.Generator(device=dev)
+    g.manual_seed(8)
+    Wc, Wa = amq.quantize(torch.randn((wl.m, wl.n), device=dev, generator=g) * wl.w_std, wl.k_w, wl.T)
+    x = torch.randn((wl.batch, wl.I), device=dev, generator=g)
+    h = torch.rand((wl.batch, wl.H), device=dev, generator=g) * 2 - 1
+    ws = amq.new_workspace(wl.I, wl.H, wl.batch, wl.k_a)
+    h1, h2 = torch.empty_like(h), torch.empty_like(h)
+    ms_default = _burst_ms(torch, lambda: amq.gru_step(Wc, Wa, None, wl.I, wl.H, x, h, wl.k_a, wl.T, ws, h_out=h1), 20)
+    ows = torch.empty((amq._lib.amq_gru_original_workspace_bytes(wl.I, wl.H, wl.batch, wl.k_a),), dtype=torch.uint8, device=dev)
+    ms_original = _burst_ms(torch, lambda: amq.gru_step_original(Wc, Wa, None, wl.I, wl.H, x, h, wl.k_a, wl.T, ows, h_out=h2), 20)
+    return {"workload": "one GRU timestep, I = H = 2048, 2/3 bits, 256 sequences: default form / original form (Cho et al.)",
+            "ms": ms_default, "ms_original_form": ms_original, "bound": "tensor+latency"}
 
 
 def table6_lines(amq, torch, dev, flush):

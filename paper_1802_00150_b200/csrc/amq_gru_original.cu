@@ -33,24 +33,26 @@ GruOrigWorkspace carve(void* base, int I, int H, int batch, int k_a)
     return w;
 }
 
-__global__ void gru_reset_kernel(const float* __restrict__ prz, const float* __restrict__ h, float* __restrict__ rh, int H, long long total)
+// (both elementwise kernels read what the preceding kernels of the stream wrote: ordinary loads after the wait)
+__global__ void gru_reset_kernel(const float* prz, const float* h, float* rh, int H, long long total)
 {
+    grid_dependency_wait();
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total) return;
     const long long b = idx / H;
     const int u = (int)(idx - b * H);
-    rh[idx] = h[idx] / (1.0f + __expf(-prz[b * 2 * H + u]));
+    rh[idx] = __ldcg(h + idx) / (1.0f + __expf(-__ldcg(prz + b * 2 * H + u)));
 }
 
-__global__ void gru_blend_kernel(const float* __restrict__ prz, const float* __restrict__ pn, const float* __restrict__ h,
-                                 float* __restrict__ h_out, int H, long long total)
+__global__ void gru_blend_kernel(const float* prz, const float* pn, const float* h, float* h_out, int H, long long total)
 {
+    grid_dependency_wait();
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total) return;
     const long long b = idx / H;
     const int u = (int)(idx - b * H);
-    const float zg = 1.0f / (1.0f + __expf(-prz[b * 2 * H + H + u]));
-    h_out[idx] = (1.0f - zg) * tanhf(pn[idx]) + zg * h[idx];
+    const float zg = 1.0f / (1.0f + __expf(-__ldcg(prz + b * 2 * H + H + u)));
+    h_out[idx] = (1.0f - zg) * tanhf(__ldcg(pn + idx)) + zg * __ldcg(h + idx);
 }
 
 }  // namespace
@@ -81,18 +83,26 @@ amq_status amq_gru_step_original(const uint32_t* Wcodes, const float* Walpha, co
     const long long total = (long long)batch * H;
     const unsigned blocks = (unsigned)((total + 255) / 256);
 
-    amq_status s = amq::launch_quantize(x, I, I, h_in, H, H, batch, k_a, T, ws.zcodes, ws.zbeta, st);
+    // every kernel of the step waits for its predecessor first thing and is launched as its programmatic dependent
+    auto product = [&](const uint32_t* Wc, const float* Wa, int m, const float* b, float* y) {
+        amq::GemmArgs a{};
+        a.Wcodes = Wc; a.Walpha = Wa; a.m = m; a.n = n; a.k_w = k_w;
+        a.xcodes = ws.zcodes; a.xbeta = ws.zbeta; a.batch = batch; a.k_a = k_a;
+        a.bias = b; a.epilogue = amq::EPI_Y; a.y = y; a.ldy = m;
+        a.overlap_with_previous = true;
+        return amq::launch_binary_gemm(a, st);
+    };
+    amq_status s = amq::launch_quantize(x, I, I, h_in, H, H, batch, k_a, T, ws.zcodes, ws.zbeta, st, true);
     if (s != AMQ_OK) return s;
-    s = amq_binary_gemm(Wcodes, Walpha, 2 * H, n, k_w, ws.zcodes, ws.zbeta, batch, k_a, bias, ws.prz, 2 * H, stream);
+    s = product(Wcodes, Walpha, 2 * H, bias, ws.prz);
     if (s != AMQ_OK) return s;
-    amq::gru_reset_kernel<<<blocks, 256, 0, st>>>(ws.prz, h_in, ws.rh, H, total);
+    AMQ_CUDA_TRY(amq::launch_kernel(amq::gru_reset_kernel, dim3(blocks), dim3(256), 0, st, true, ws.prz, h_in, ws.rh, H, total));
     AMQ_LAUNCH_CHECK();
-    s = amq::launch_quantize(x, I, I, ws.rh, H, H, batch, k_a, T, ws.zcodes, ws.zbeta, st);
+    s = amq::launch_quantize(x, I, I, ws.rh, H, H, batch, k_a, T, ws.zcodes, ws.zbeta, st, true);
     if (s != AMQ_OK) return s;
-    s = amq_binary_gemm(Wcodes + (size_t)2 * H * k_w * wpr, Walpha + (size_t)2 * H * k_w, H, n, k_w, ws.zcodes, ws.zbeta,
-                        batch, k_a, bias ? bias + 2 * H : nullptr, ws.pn, H, stream);
+    s = product(Wcodes + (size_t)2 * H * k_w * wpr, Walpha + (size_t)2 * H * k_w, H, bias ? bias + 2 * H : nullptr, ws.pn);
     if (s != AMQ_OK) return s;
-    amq::gru_blend_kernel<<<blocks, 256, 0, st>>>(ws.prz, ws.pn, h_in, h_out, H, total);
+    AMQ_CUDA_TRY(amq::launch_kernel(amq::gru_blend_kernel, dim3(blocks), dim3(256), 0, st, true, ws.prz, ws.pn, h_in, h_out, H, total));
     AMQ_LAUNCH_CHECK();
     return AMQ_OK;
 }
