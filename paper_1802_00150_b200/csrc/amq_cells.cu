@@ -82,7 +82,7 @@ amq_status enqueue_sequence(const CellCall& c, const CellWorkspace& ws, const fl
 {
     const size_t state_bytes = (size_t)c.batch * c.H * sizeof(float);
     const bool persistent = steps > 0 && use_persistent(c);
-    AMQ_CUDA_TRY(cudaMemsetAsync(ws.status, 0, 256 + ((persistent && steps > 1) ? (size_t)2 * c.H * 8 : 0), st));
+    AMQ_CUDA_TRY(cudaMemsetAsync(ws.status, 0, 256 + ((persistent && steps > 1) ? ws.hx_bytes : 0), st));
     if (persistent)
         return enqueue_persistent(c, ws, x_seq, steps, h0, c0, h_seq, h_last, c_last, st);
     if (!c.gru) AMQ_CUDA_TRY(cudaMemcpyAsync(ws.c, c0, state_bytes, cudaMemcpyDeviceToDevice, st));

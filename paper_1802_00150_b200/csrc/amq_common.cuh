@@ -37,14 +37,21 @@ inline bool valid_k(int k) { return k >= 1 && k <= AMQ_MAX_K; }
 inline int words_per_row(int n) { return 4 * ((n + 127) / 128); }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Layout of a cell workspace: [status block][z codes][z coefficients][h ping][h pong][c].
+// Copies of the h exchange buffer of the persistent batch-1 kernel: every producer writes each copy, a CTA polls
+// copy blockIdx.x % copies, which spreads the polling over that many times more L2 lines.
+constexpr int PERSISTENT_EXCHANGE_COPIES = 8;
+// words per copy: H rounded up to whole 128-byte lines, so every copy starts on a line
+inline size_t persistent_exchange_stride(int H) { return ((size_t)H + 15) / 16 * 16; }
+
+// Layout of a cell workspace: [status block][exchange words][z codes][z coefficients][h ping][h pong][c].
 struct CellWorkspace {
     uint32_t* status;   // 64 words: [0] status, [1..] barrier counters
     uint32_t* zcodes;   // [batch][k_a][wpr]
     float* zbeta;       // [batch][k_a]
     float* h[2];        // [batch][H] each
     float* c;           // [batch][H]
-    unsigned long long* hx;   // [2][H] exchange words {fp32 bits, step tag} of the persistent kernel
+    unsigned long long* hx;   // [2][copies][H] exchange words {fp32 bits, step tag} of the persistent kernel
+    size_t hx_bytes;
     size_t bytes;
 };
 
@@ -55,7 +62,9 @@ inline CellWorkspace carve_cell_workspace(void* base, int I, int H, int batch, i
     size_t off = 0;
     w.status = reinterpret_cast<uint32_t*>(p + off);            off += 256;
     // the exchange words directly behind the status words: one memset clears both before a sequence
-    w.hx = reinterpret_cast<unsigned long long*>(p + off);      off += round_up((size_t)2 * H * 8, 256);
+    w.hx = reinterpret_cast<unsigned long long*>(p + off);
+    w.hx_bytes = batch == 1 ? round_up((size_t)2 * PERSISTENT_EXCHANGE_COPIES * persistent_exchange_stride(H) * 8, 256) : 0;   // batch 1 only
+    off += w.hx_bytes;
     w.zcodes = reinterpret_cast<uint32_t*>(p + off);            off += round_up((size_t)batch * k_a * words_per_row(I + H) * 4, 256);
     w.zbeta = reinterpret_cast<float*>(p + off);                off += round_up((size_t)batch * k_a * 4, 256);
     w.h[0] = reinterpret_cast<float*>(p + off);                 off += round_up((size_t)batch * H * 4, 256);
@@ -146,6 +155,7 @@ amq_status launch_rnn_persistent(const uint32_t* Wcodes, const float* Walpha, co
                                  int I, int H, int k_w, int k_a, int T, bool gru,
                                  const float* x_seq, int steps, const float* h0, const float* c0,
                                  float* h_seq, float* h_last, float* c_last,
-                                 unsigned long long* hx, uint32_t* status, cudaStream_t st);
+                                 unsigned long long* hx, uint32_t* status, cudaStream_t st,
+                                 unsigned poll_limit = 0, unsigned tag_bias = 0);
 
 }  // namespace amq

@@ -28,7 +28,7 @@ __global__ void __launch_bounds__(128)
 quantize_rows_consecutive_kernel(const float* __restrict__ x, int ldx, int rows, int n, int T,
                                  uint32_t* __restrict__ codes, float* __restrict__ coeffs)
 {
-    __shared__ QuantScratch<K> scratch[4];
+    __shared__ QuantScratch<K, 1> scratch[4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int row = blockIdx.x * (blockDim.x >> 5) + warp;
     if (row >= rows) return;
@@ -51,7 +51,7 @@ quantize_rows_consecutive_kernel(const float* __restrict__ x, int ldx, int rows,
     }
     float alpha[K];
     uint32_t bits[K];
-    quantize_group<K, 32, false>(w, valid, n, T, alpha, bits, scratch[warp]);
+    quantize_group<K, 32, 1>(w, valid, n, T, alpha, bits, scratch[warp]);
     const int wpr = 4 * ((n + 127) / 128);
     if (lane < wpr) {
 #pragma unroll
@@ -65,12 +65,14 @@ quantize_rows_consecutive_kernel(const float* __restrict__ x, int ldx, int rows,
     }
 }
 
-// K bits, EPT elements per thread.  MULTI: one row per CTA (blockDim.x threads); else one row per warp.
+// K bits, EPT elements per thread.  MULTI: one row per CTA (blockDim.x <= 256 threads); else one row per warp.
 template <int K, int EPT, bool MULTI>
 __global__ void __launch_bounds__(256)
 quantize_kernel(RowSource src, int rows, int n, int T, uint32_t* __restrict__ codes, float* __restrict__ coeffs)
 {
-    __shared__ QuantScratch<K> scratch[MULTI ? 1 : 4];
+    constexpr int NW = MULTI ? 8 : 1;
+    __shared__ QuantScratch<K, NW> scratch[MULTI ? 1 : 4];
+    if (MULTI) quant_scratch_init(scratch[0]);
     grid_dependency_wait();             // launched early behind a product kernel: its state output must be complete
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -91,7 +93,7 @@ quantize_kernel(RowSource src, int rows, int n, int T, uint32_t* __restrict__ co
 
     float alpha[K];
     uint32_t bits[K];
-    quantize_group<K, EPT, MULTI>(w, valid, n, T, alpha, bits, scratch[MULTI ? 0 : warp]);
+    quantize_group<K, EPT, NW>(w, valid, n, T, alpha, bits, scratch[MULTI ? 0 : warp]);
 
     const int wpr = 4 * ((n + 127) / 128);
     pack_group<K, EPT>(bits, lane, MULTI ? warp : 0, G >> 5, wpr, codes + (size_t)row * K * wpr);

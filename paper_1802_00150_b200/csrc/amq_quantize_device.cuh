@@ -2,10 +2,10 @@
 // row quantizer kernel and by the persistent recurrent kernel, which quantizes [x ; h] in place.
 //
 // A "group" of threads owns one vector; every thread holds EPT of its elements in registers (which ones is
-// the caller's choice).  Data-parallel form of Algorithm 1 ("maintaining a mask vector ... operate BST for
-// all entries simultaneously", Sec. 3): every element descends the tree over the 2^k - 1 midpoints of the
-// ascending level table with k compares and predicated selects of the next midpoint (no branches), and the
-// leaf index looks the sign pattern up in one small bit table per plane.
+// the caller's choice).  Algorithm 1 is evaluated in its data-parallel form (the remark on operating on all
+// entries at once, Sec. 3): every element descends the tree over the 2^k - 1 midpoints of the ascending level
+// table with k compares and predicated selects of the next midpoint (no branches), and the leaf index looks
+// the sign pattern up in one small bit table per plane.
 //
 // Instruction economy of the inner loops (they decide the throughput of bulk quantization): inputs are
 // canonicalised (-0.0 -> +0.0), after which "r >= 0" is exactly "sign bit clear" for every residue the
@@ -16,14 +16,17 @@
 // cleared at the end, they add nothing to B^T w, the Gram matrix is counted on masked words, and their known
 // contribution to the greedy |r| sums (all of them follow the trajectory of a zero element) is subtracted.
 //
-// Arithmetic: sums over the vector are fp32 (per thread, then a fixed butterfly / warp order, so results
-// are reproducible run to run); the Gram matrix B^T B is exact integer arithmetic; the k x k solve is
-// fp64; levels, midpoints and comparisons are fp32.
+// Arithmetic: sums over the vector are fp32 (per thread, then a fixed butterfly over the warp, then the
+// per-warp partials in a fixed tree, so results are reproducible run to run); the Gram matrix B^T B is exact
+// integer arithmetic; the k x k solve is fp64 for k >= 3 and error-compensated fp32 for k = 2 (the products
+// n c_i and g c_j are split exactly with fused multiply-adds, so cancellation costs nothing); levels,
+// midpoints and comparisons are fp32.
 //
-// When the group is a whole CTA, the per-vector scalar work (cross-warp totals, the k x k solve, the
-// sorted level table) is done once by warp 0 and handed to the other warps through shared memory, rather
-// than repeated by every warp: in the persistent kernel the quantizer sits on the latency path of each
-// timestep, and issue slots, not arithmetic, are what it runs out of.
+// When the group is a whole CTA, a reduction costs ONE barrier: lane 0 of every warp leaves the warp's
+// partial sums in shared memory, and after the barrier every thread adds up all partials itself and
+// repeats the per-vector scalar work (solve, sorted level table) redundantly.  In the recurrent kernels the
+// quantizer sits on the latency path of each timestep, and a second barrier plus a round trip through
+// shared memory for "one warp computes, all read" costs more than the repeated arithmetic.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -33,30 +36,34 @@ namespace amq {
 
 constexpr int QUANT_MAX_WARPS = 16;
 
-template <int K>
-struct QuantOut {                       // what the leader warp publishes after a reduction
-    float alpha[K];
-    float thr[(1 << K) - 1];
-    uint32_t plane[K];                  // bit p of plane[i]: sign (1 = +1) of plane i at sorted level p
-};
-
-// Shared-memory scratch of one group (a warp, or a CTA of up to 16 warps).
-template <int K>
-struct QuantScratch {
+// Shared-memory scratch of one group of NW warps (NW = 1: a single warp, which needs the level scratch only).
+template <int K, int NW>
+struct __align__(16) QuantScratch {
     static constexpr int V = 1 + K + K * (K - 1) / 2;
-    static constexpr int STRIDE = V + (V & 1);
-    float red[2][QUANT_MAX_WARPS][STRIDE];   // per-warp partial sums, double-buffered by reduction parity
-    QuantOut<K> out[2];
-    float level[1 << K];
-    int code[1 << K];
+    static constexpr int SLOTS = NW > 1 ? ((NW + 3) / 4) * 4 : 4;
+    float red[2][V][SLOTS];             // [reduction parity][value][warp]: per-warp partial sums
+    float level[NW][1 << K];            // per-warp scratch of the level sort (k >= 3)
+    int code[NW][1 << K];
 };
 
-// Totals over the group of VF floats and VI ints (ints are carried exactly).  Returns true in the threads
-// that hold the totals afterwards: every thread when the group is one warp; the threads of warp 0 when the
-// group is the CTA (MULTI).  In the MULTI case the caller must publish what the others need and
-// __syncthreads() before they read it.
-template <int VF, int VI, int K, bool MULTI>
-__device__ __forceinline__ bool group_totals(float (&f)[VF], int (&iv)[VI > 0 ? VI : 1], QuantScratch<K>& sc, int parity)
+// To be called once by every thread of a CTA-wide group before its first quantize_group (no barrier needed
+// afterwards): partial-sum slots of warps that do not exist are read as zeros by every reduction.
+template <int K, int NW>
+__device__ __forceinline__ void quant_scratch_init(QuantScratch<K, NW>& sc)
+{
+    constexpr int V = QuantScratch<K, NW>::V, SLOTS = QuantScratch<K, NW>::SLOTS;
+    const int warps = blockDim.x >> 5;
+    float* flat = &sc.red[0][0][0];
+    for (int idx = threadIdx.x; idx < 2 * V * SLOTS; idx += blockDim.x)
+        if ((idx % SLOTS) >= warps) flat[idx] = 0.0f;
+}
+
+// Totals over the group of VF floats and VI ints (ints are carried exactly); every thread of the group holds
+// them afterwards.  NW > 1: the group is the CTA and the call contains exactly one CTA barrier; when `flag`
+// is given, that barrier also ORs *flag over the CTA (every thread gets the result).
+template <int VF, int VI, int K, int NW>
+__device__ __forceinline__ void group_totals(float (&f)[VF], int (&iv)[VI > 0 ? VI : 1], QuantScratch<K, NW>& sc,
+                                             int parity, int* flag = nullptr)
 {
 #pragma unroll
     for (int i = 0; i < VF; ++i) {
@@ -65,35 +72,44 @@ __device__ __forceinline__ bool group_totals(float (&f)[VF], int (&iv)[VI > 0 ? 
     }
 #pragma unroll
     for (int i = 0; i < VI; ++i) iv[i] = __reduce_add_sync(0xffffffffu, iv[i]);
-    if (!MULTI) return true;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+    if (NW == 1) return;
+    constexpr int SLOTS = QuantScratch<K, NW>::SLOTS;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (lane == 0) {
-        float* mine = sc.red[parity][warp];
 #pragma unroll
-        for (int i = 0; i < VF; ++i) mine[i] = f[i];
+        for (int i = 0; i < VF; ++i) sc.red[parity][i][warp] = f[i];
 #pragma unroll
-        for (int i = 0; i < VI; ++i) mine[VF + i] = __int_as_float(iv[i]);
+        for (int i = 0; i < VI; ++i) sc.red[parity][VF + i][warp] = __int_as_float(iv[i]);
     }
-    __syncthreads();
-    if (warp != 0) return false;
-    // warp 0: lane l holds the partials of warp l; sum over lanes in a fixed butterfly
-    const bool have = lane < warps;
-    const float* src = sc.red[parity][have ? lane : 0];
+    if (flag) *flag = __syncthreads_or(*flag);
+    else __syncthreads();
+    // every thread: the partials of all warps, added in a fixed tree (slots of absent warps hold zeros)
 #pragma unroll
     for (int i = 0; i < VF; ++i) {
-        float v = have ? src[i] : 0.0f;
+        float tot = 0.0f;
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-        f[i] = v;
+        for (int q = 0; q < SLOTS / 4; ++q) {
+            const float4 v = *reinterpret_cast<const float4*>(&sc.red[parity][i][4 * q]);
+            const float s = (v.x + v.y) + (v.z + v.w);
+            tot = (q == 0) ? s : tot + s;
+        }
+        f[i] = tot;
     }
 #pragma unroll
-    for (int i = 0; i < VI; ++i) iv[i] = __reduce_add_sync(0xffffffffu, have ? __float_as_int(src[VF + i]) : 0);
-    return true;
+    for (int i = 0; i < VI; ++i) {
+        int tot = 0;
+#pragma unroll
+        for (int q = 0; q < SLOTS / 4; ++q) {
+            const int4 v = *reinterpret_cast<const int4*>(&sc.red[parity][VF + i][4 * q]);
+            tot += (v.x + v.y) + (v.z + v.w);
+        }
+        iv[i] = tot;
+    }
 }
 
 // Least-squares solve of Eq. 5, G a = c with G = B^T B (G_ii = n, integer off-diagonals in gram[], row
-// major upper triangle) in fp64.  Leaves `a` untouched and returns false when a pivot of Gaussian
-// elimination with partial pivoting falls below 1e-9 * n (reading for a singular system: skip the refit).
+// major upper triangle).  Leaves `a` untouched and returns false when a pivot of Gaussian elimination with
+// partial pivoting falls below 1e-9 * n (reading for a singular system: skip the refit).
 template <int K>
 __device__ __forceinline__ bool solve_refit(const float (&c)[K], const int (&gram)[K > 1 ? K * (K - 1) / 2 : 1], int n,
                                             float (&a)[K])
@@ -105,17 +121,18 @@ __device__ __forceinline__ bool solve_refit(const float (&c)[K], const int (&gra
     }
     if (K == 2) {
         // pivots of the elimination are n and (n^2 - g^2) / n: the second is below 1e-9 n only when the
-        // integer n^2 - g^2 is zero (n <= 8192), i.e. b_1 = +-b_2
+        // integer n^2 - g^2 is zero (n <= 8192), i.e. b_1 = +-b_2.  Cramer's rule on the exact integers; each
+        // numerator n c_i - g c_j is formed without cancellation error: t = fl(g c_j), e = g c_j - t exactly
+        // (fused multiply-add), fl(n c_i - t) rounds once relative to the RESULT, then e is taken off.
         const int g = gram[0];
-        const int det = n * n - g * g;                       // |.| <= 2^26: exact in int and in double
+        const int det = n * n - g * g;                       // |.| <= 2^26: exact in int
         if (det == 0) return false;
-        const double dd = (double)det;
-        double r = (double)__frcp_rn((float)det);            // fp32 seed, one Newton step in fp64
-        r = r * (2.0 - dd * r);
-        r = r * (2.0 - dd * r);
-        const double c0 = (double)c[0], c1 = (double)c[1], dn = (double)n, dg = (double)g;
-        a[0] = (float)((dn * c0 - dg * c1) * r);
-        a[1] = (float)((dn * c1 - dg * c0) * r);
+        const float fn = (float)n, fg = (float)g;            // exact (<= 8192)
+        const float rdet = __fdividef(1.0f, (float)det);     // |det| <= 2^26: in range of the fast reciprocal
+        const float t0 = fg * c[1], e0 = fmaf(fg, c[1], -t0);
+        const float t1 = fg * c[0], e1 = fmaf(fg, c[0], -t1);
+        a[0] = (fmaf(fn, c[0], -t0) - e0) * rdet;
+        a[1] = (fmaf(fn, c[1], -t1) - e1) * rdet;
         return true;
     }
     double G[K][K + 1];
@@ -165,40 +182,57 @@ __device__ __forceinline__ bool solve_refit(const float (&c)[K], const int (&gra
     return true;
 }
 
+// Per-plane bit tables of the sorted code table: bit p of plane[i] = sign (1 = +1) of plane i at level p.
+template <int K>
+__device__ __forceinline__ void planes_from_table(unsigned long long table, uint32_t (&plane)[K])
+{
+#pragma unroll
+    for (int i = 0; i < K; ++i) plane[i] = 0u;
+#pragma unroll
+    for (int p = 0; p < (1 << K); ++p) {
+        const uint32_t code = (uint32_t)(table >> (4 * p)) & 15u;
+#pragma unroll
+        for (int i = 0; i < K; ++i) plane[i] |= ((code >> (K - 1 - i)) & 1u) << p;
+    }
+}
+
 // Ascending level table of the 2^K values sum_i +-alpha_i, ordered by (value, code index), plane 0 the most
-// significant code bit.  Produces the 2^K - 1 midpoints and the codes packed 4 bits per table position.
-// Executed by one full warp (K >= 3 uses its lanes and __syncwarp).
+// significant code bit.  Produces the 2^K - 1 midpoints and, per plane, the signs along the table (bit p of
+// plane[i]: sign, 1 = +1, of plane i at sorted level p).
+// Executed by one full warp (K >= 3 uses its lanes, __syncwarp and the warp's own scratch rows).
 template <int K>
 __device__ __forceinline__ void level_table(const float (&alpha)[K], int lane, float (&thr)[(1 << K) - 1],
-                                            unsigned long long& table, QuantScratch<K>& sc)
+                                            uint32_t (&plane)[K], float* sc_level, int* sc_code)
 {
     constexpr int M = 1 << K;
+    unsigned long long table = 0ull;          // codes packed 4 bits per table position (K != 2)
     if (K == 1) {
         // levels -a, +a (or swapped when a < 0); the midpoint is 0 either way
         thr[0] = (-alpha[0] + alpha[0]) * 0.5f;
         table = (alpha[0] < 0.0f) ? 0x01ull : 0x10ull;
+        planes_from_table<K>(table, plane);
         return;
     }
     if (K == 2) {
-        float v[4];
-        int c[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            float s = 0.0f;
-            s += (q & 2) ? alpha[0] : -alpha[0];
-            s += (q & 1) ? alpha[1] : -alpha[1];
-            v[q] = s; c[q] = q;
+        // The four levels +-a +-b in closed form.  With A = |a|, B = |b| the ascending values are
+        // -(A+B), -|A-B|, +|A-B|, A+B, so the midpoints are -(fl(A+B) + |fl(A-B)|)/2, 0 and its negative
+        // (exactly what sorting the four rounded sums gives).  In terms of the magnitudes the sign patterns
+        // come in the order (-,-) (-,+) (+,-) (+,+) when A > B and (-,-) (+,-) (-,+) (+,+) when A < B; a
+        // negative coefficient flips its own bit of every code.  Equal values are ordered by code index:
+        // A == B ties the two middle levels (the first order is the ascending one unless a < 0); a coefficient
+        // that is zero, or vanishes against the other in fp32, ties the outer pairs, and its bit then ascends.
+        const float a = alpha[0], b = alpha[1];
+        const float A = fabsf(a), B = fabsf(b);
+        const float d = A - B;
+        const float t0 = -0.5f * ((A + B) + fabsf(d));
+        thr[0] = t0; thr[1] = 0.0f; thr[2] = -t0;
+        bool sa = a < 0.0f, sb = b < 0.0f;
+        const bool first = d > 0.0f || (d == 0.0f && !sa);
+        if ((A + B) == fabsf(d)) {            // the smaller coefficient vanishes in the sums: its sign orders nothing
+            if (first) sb = false; else sa = false;
         }
-#define AMQ_CSWAP(x, y)                                                                   \
-        if (v[x] > v[y] || (v[x] == v[y] && c[x] > c[y])) {                               \
-            const float tv = v[x]; v[x] = v[y]; v[y] = tv;                                \
-            const int tc = c[x]; c[x] = c[y]; c[y] = tc;                                  \
-        }
-        AMQ_CSWAP(0, 1) AMQ_CSWAP(2, 3) AMQ_CSWAP(0, 2) AMQ_CSWAP(1, 3) AMQ_CSWAP(1, 2)
-#undef AMQ_CSWAP
-#pragma unroll
-        for (int p = 0; p < 3; ++p) thr[p] = (v[p] + v[p + 1]) * 0.5f;
-        table = (unsigned long long)(c[0] | (c[1] << 4) | (c[2] << 8) | (c[3] << 12));
+        plane[0] = (first ? 0xCu : 0xAu) ^ (sa ? 0xFu : 0u);      // bit p: sign of plane 0 at level p
+        plane[K - 1] = (first ? 0xAu : 0xCu) ^ (sb ? 0xFu : 0u);
         return;
     }
     // K >= 3: lane c < 2^K ranks its own level among all, through shared memory
@@ -215,29 +249,15 @@ __device__ __forceinline__ void level_table(const float (&alpha)[K], int lane, f
             for (int i = 0; i < K; ++i) v += ((c >> (K - 1 - i)) & 1) ? alpha[i] : -alpha[i];
             rank += (v < mine || (v == mine && c < lane)) ? 1 : 0;
         }
-        sc.level[rank] = mine;
-        sc.code[rank] = lane;
+        sc_level[rank] = mine;
+        sc_code[rank] = lane;
     }
     __syncwarp();
-    table = 0ull;
 #pragma unroll
-    for (int p = 0; p < M - 1; ++p) thr[p] = (sc.level[p] + sc.level[p + 1]) * 0.5f;
+    for (int p = 0; p < M - 1; ++p) thr[p] = (sc_level[p] + sc_level[p + 1]) * 0.5f;
 #pragma unroll
-    for (int p = 0; p < M; ++p) table |= (unsigned long long)sc.code[p] << (4 * p);
-}
-
-// Per-plane bit tables of the sorted code table: bit p of plane[i] = sign (1 = +1) of plane i at level p.
-template <int K>
-__device__ __forceinline__ void planes_from_table(unsigned long long table, uint32_t (&plane)[K])
-{
-#pragma unroll
-    for (int i = 0; i < K; ++i) plane[i] = 0u;
-#pragma unroll
-    for (int p = 0; p < (1 << K); ++p) {
-        const uint32_t code = (uint32_t)(table >> (4 * p)) & 15u;
-#pragma unroll
-        for (int i = 0; i < K; ++i) plane[i] |= ((code >> (K - 1 - i)) & 1u) << p;
-    }
+    for (int p = 0; p < M; ++p) table |= (unsigned long long)sc_code[p] << (4 * p);
+    planes_from_table<K>(table, plane);
 }
 
 // Algorithm 1 for one element: index of the leaf (sorted level) the descent over the midpoints reaches.
@@ -270,25 +290,32 @@ __device__ __forceinline__ int bst_leaf(float x, const float (&thr)[(1 << K) - 1
 }
 
 // Quantize the vector held in w[] (positions past the end of the vector must hold 0 and have their bit
-// clear in `valid`; `padding` is their number over the whole group).  On return alpha[i] are the
-// coefficients and bit j of bits[i] is the sign (1 = +1) of element j of this thread in plane i.
+// clear in `valid`).  NW = 1: the group is the calling warp; NW > 1: the group is the whole CTA of up to NW
+// warps (quant_scratch_init must have run).  On return alpha[i] are the coefficients and bit j of bits[i] is
+// the sign (1 = +1) of element j of this thread in plane i.
 //
 // The greedy step needs k dependent reductions (each coefficient is the mean |residue| left by the
 // previous one, Eq. 3-4); the sign plane of the last greedy bit does not depend on its own coefficient,
 // so that last reduction travels together with the sums of the first refit (Eq. 5): k + T - 1 group
-// reductions in all for T >= 1, with the values Algorithm 2 prescribes.
-template <int K, int EPT, bool MULTI>
+// reductions in all for T >= 1, with the values Algorithm 2 prescribes; each is one CTA barrier when the
+// group is the CTA.  `flag` (CTA groups only, may be NULL): ORed over the CTA by the first of those barriers,
+// so a caller can fold a "some thread gave up waiting for its input" vote into it; `parity` (CTA groups
+// only): which half of the double-buffered partial-sum scratch the first reduction uses, updated on return,
+// so that consecutive calls keep alternating.
+template <int K, int EPT, int NW>
 __device__ __forceinline__ void quantize_group(const float (&w_in)[EPT], uint32_t valid, int n, int T,
-                                               float (&alpha)[K], uint32_t (&bits)[K], QuantScratch<K>& sc)
+                                               float (&alpha)[K], uint32_t (&bits)[K], QuantScratch<K, NW>& sc,
+                                               int* flag = nullptr, int* parity_io = nullptr)
 {
     constexpr int M = 1 << K;
     constexpr int NG = K * (K - 1) / 2;
     constexpr uint32_t SIGN = 0x80000000u;
     const int lane = threadIdx.x & 31;
+    const int slot = NW > 1 ? (int)(threadIdx.x >> 5) : 0;
     const int nvalid = __popc(valid);
     const float inv_n = 1.0f / (float)n;
-    const float padding = (float)((MULTI ? (int)blockDim.x : 32) * EPT - n);     // zero elements past the end
-    int parity = 0;
+    const float padding = (float)((NW > 1 ? (int)blockDim.x : 32) * EPT - n);    // zero elements past the end
+    int parity = parity_io ? *parity_io : 0;
 
     float w[EPT];
 #pragma unroll
@@ -317,14 +344,10 @@ __device__ __forceinline__ void quantize_group(const float (&w_in)[EPT], uint32_
             if (i == K - 1 && T > 0) { last_abs = part; alpha[i] = 0.0f; break; }
             float tot[1] = {part};
             int none[1] = {0};
-            const bool leader = group_totals<1, 0, K, MULTI>(tot, none, sc, parity);
-            float a = (tot[0] - padding * fabsf(rho)) * inv_n;
-            if (MULTI) {
-                if (leader && lane == 0) sc.out[parity].alpha[0] = a;
-                __syncthreads();
-                a = sc.out[parity].alpha[0];
-            }
+            group_totals<1, 0, K, NW>(tot, none, sc, parity, flag);
+            flag = nullptr;
             parity ^= 1;
+            const float a = (tot[0] - padding * fabsf(rho)) * inv_n;
             alpha[i] = a;
             const uint32_t ab = __float_as_uint(a);               // a >= 0
             rho -= __uint_as_float(ab | (__float_as_uint(rho) & SIGN));
@@ -351,35 +374,19 @@ __device__ __forceinline__ void quantize_group(const float (&w_in)[EPT], uint32_
                     gram[q++] = nvalid - 2 * __popc((bits[i] ^ bits[j]) & valid);
             if (NG == 0) gram[0] = 0;
         }
-        const bool leader = group_totals<1 + K, NG, K, MULTI>(fsum, gram, sc, parity);
+        group_totals<1 + K, NG, K, NW>(fsum, gram, sc, parity, flag);
+        flag = nullptr;
+        parity ^= 1;
         float thr[M - 1];
         uint32_t plane[K];
-        if (leader) {
+        {
             if (it == 0) alpha[K - 1] = (fsum[0] - padding * fabsf(rho)) * inv_n;   // the last greedy coefficient
             float c[K];
 #pragma unroll
             for (int i = 0; i < K; ++i) c[i] = fsum[1 + i];
             solve_refit<K>(c, gram, n, alpha);
-            unsigned long long table = 0ull;
-            level_table<K>(alpha, lane, thr, table, sc);
-            planes_from_table<K>(table, plane);
-            if (MULTI && lane == 0) {
-                QuantOut<K>& o = sc.out[parity];
-#pragma unroll
-                for (int i = 0; i < K; ++i) { o.alpha[i] = alpha[i]; o.plane[i] = plane[i]; }
-#pragma unroll
-                for (int p = 0; p < M - 1; ++p) o.thr[p] = thr[p];
-            }
+            level_table<K>(alpha, lane, thr, plane, sc.level[slot], sc.code[slot]);
         }
-        if (MULTI) {
-            __syncthreads();
-            const QuantOut<K>& o = sc.out[parity];
-#pragma unroll
-            for (int i = 0; i < K; ++i) { alpha[i] = o.alpha[i]; plane[i] = o.plane[i]; }
-#pragma unroll
-            for (int p = 0; p < M - 1; ++p) thr[p] = o.thr[p];
-        }
-        parity ^= 1;
         last_abs = 0.0f;
 
         // Algorithm 1 for every element; the sums B^T w of the next refit are taken in the same pass
@@ -400,6 +407,7 @@ __device__ __forceinline__ void quantize_group(const float (&w_in)[EPT], uint32_
 #pragma unroll
         for (int i = 0; i < K; ++i) bits[i] = pos_bits[i] & valid;
     }
+    if (parity_io) *parity_io = parity;
 }
 
 // Pack the sign bits of a group into words: word (j * G/32 + warp-in-group) of plane i is the ballot

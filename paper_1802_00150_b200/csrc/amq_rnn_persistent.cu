@@ -1,19 +1,24 @@
 // Persistent, weight-stationary kernel for a batch-1 quantized LSTM / GRU sequence (Eq. 6 repeated over
-// time; "RNNs can only be executed sequentially", Sec. 1).
+// time; timestep t + 1 consumes h_t, Sec. 1, so a sequence is one dependency chain).
 //
 // The hidden units are split over the CTAs of one co-resident (cooperative) grid; every CTA keeps the
 // packed planes of its own gate rows in shared memory for the whole sequence.  A timestep is, in every
 // CTA: gather z = [x_t ; h_{t-1}], quantize it on-line (Algorithm 2, all CTAs redundantly, so that one
-// exchange per step is enough), XOR + bit-count its planes against the resident rows (Appendix A), fold
-// the partials with the row-wise coefficients (Sec. 4), apply the gates and publish the new h slice.
+// exchange per step is enough; one CTA barrier per reduction), pack the planes (one more barrier), then
+// one warp per hidden unit XORs and bit-counts the planes against the unit's resident rows (Appendix A),
+// folds the partials with the row-wise coefficients (Sec. 4), applies the gates and publishes the new h
+// value, all inside the warp with shuffles; the other warps are already gathering for the next step.
 //
 // Exchange of h between CTAs: each value travels as one 64-bit word {fp32 bits, step tag}, written with
 // a single relaxed gpu-scope store and polled with relaxed gpu-scope loads; a consumer accepts a word
 // when its tag equals the step it is gathering for, so value and "ready" flag arrive together and no
-// separate barrier, fence or atomic counter is on the critical path.  Two buffers alternate by step
-// parity: a CTA can only run one step ahead of the slowest one (it needs every slice of the previous
-// step), so a buffer is never overwritten while someone still reads it.  Every poll is bounded; when
-// it runs out the CTA records AMQ_ERR_TIMEOUT in the workspace status word and leaves.
+// separate barrier, fence or atomic counter is on the critical path.  Every producer writes its word to
+// several copies of the exchange buffer and a CTA polls the copy blockIdx.x % copies: all CTAs polling the
+// same few cache lines queue up at the L2 slices that hold them, and the queueing, not the distance, was
+// most of the exchange latency.  Two buffers alternate by step parity: a CTA can only run one step ahead
+// of the slowest one (it needs every slice of the previous step), so a buffer is never overwritten while
+// someone still reads it.  Every poll is bounded; when it runs out the CTA records AMQ_ERR_TIMEOUT in the
+// workspace status word and leaves (the vote is folded into the first barrier of the quantizer).
 #include "amq_common.cuh"
 #include "amq_quantize_device.cuh"
 
@@ -21,7 +26,6 @@ namespace amq {
 
 namespace {
 
-constexpr int NT = 512;                  // threads per CTA
 constexpr unsigned POLL_LIMIT = 1u << 20;
 
 struct PersistArgs {
@@ -29,16 +33,30 @@ struct PersistArgs {
     int I, H, k_w, T, steps;
     const float* x_seq; const float* h0; const float* c0;
     float* h_seq; float* h_last; float* c_last;
-    unsigned long long* hx;              // [2][H] exchange words
+    unsigned long long* hx;              // [2][copies][hx_stride] exchange words
+    size_t hx_stride;                    // H rounded up to whole 128-byte lines
+    int vec_ok;                          // I % EPT == 0, H even, x_seq 16-byte aligned: vector loads, no thread straddles x | h
     uint32_t* status;
     int upc;                             // hidden units per CTA
     int wpr;
+    int copies;                          // copies of the exchange buffer (1..32)
+    unsigned poll_limit;                 // iterations after which a gather gives up
+    unsigned tag_bias;                   // added to the tag a gather expects (0; nonzero only in the self-test of the
+                                         // give-up path, where no word can ever match)
 };
 
 __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p)
 {
     unsigned long long v;
     asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// two adjacent exchange words with one 16-byte load (each word is validated on its own by its tag)
+__device__ __forceinline__ ulonglong2 ld_relaxed_v2_u64(const unsigned long long* p)
+{
+    ulonglong2 v;
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "l"(p) : "memory");
     return v;
 }
 
@@ -56,15 +74,11 @@ __device__ __forceinline__ int popc4(uint4 a, uint4 b)
     return __popc(a.x ^ b.x) + __popc(a.y ^ b.y) + __popc(a.z ^ b.z) + __popc(a.w ^ b.w);
 }
 
-// Lanes per plane-row in the product phase: the largest power of two that still gives every plane-row of
-// the CTA its own segment in one pass, at most one lane per 128-bit chunk, at most a warp.
-__host__ __device__ inline int product_segment(int PR, int CH)
+// Lanes per plane-row in the product phase: a warp holds all plane-rows of one hidden unit (gates x k_w <= 16),
+// each owned by a segment of SEG lanes (a power of two).
+__host__ __device__ inline int product_segment(int rows_per_unit)
 {
-    int cap = 1;
-    while (cap < CH && cap < 32) cap <<= 1;
-    int seg = 1;
-    while (seg * 2 <= cap && seg * 2 * PR <= NT) seg <<= 1;
-    return seg;
+    return rows_per_unit <= 4 ? 8 : (rows_per_unit <= 8 ? 4 : 2);
 }
 
 // Row stride of the resident planes in 16-byte units: segments narrower than a quarter-warp are skewed so
@@ -80,32 +94,36 @@ __host__ __device__ inline int product_row_stride(int CH, int SEG)
 #define AMQ_PHASE(i) do { } while (0)
 #endif
 
-template <int KA, int EPT, bool GRU>
+template <int KA, int EPT, bool GRU, int NT>
 __global__ void __launch_bounds__(NT, 1)
 rnn_persistent_kernel(PersistArgs a)
 {
+    constexpr int NW = NT / 32;
     constexpr int GATES = GRU ? 3 : 4;
     constexpr int PARTS = GRU ? 2 : 1;    // GRU keeps the product in two column segments, [0,I) and [I,n)
+    static_assert(EPT == 8 || EPT == 16, "a thread's sign bits are stored as one byte or one half-word");
     extern __shared__ __align__(16) unsigned char smem_raw[];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = a.I + a.H, wpr = a.wpr, CH = wpr >> 2, k_w = a.k_w;
-    const int upc = a.upc, rows = upc * GATES, PR = rows * k_w;
+    const int upc = a.upc, RPU = GATES * k_w, PR = upc * RPU;
     const int u0 = blockIdx.x * upc;
 
-    // product role: segments of SEG lanes share a plane-row; lane c of a segment owns chunks c, c + SEG, ..
-    const int SEG = product_segment(PR, CH), RS = product_row_stride(CH, SEG);
-    const int NSEG = NT / SEG, seg = tid / SEG, chunk = tid % SEG;
-    const int pr_iters = (PR + NSEG - 1) / NSEG;
+    // product role: lane = (plane-row within the unit) * SEG + chunk; lane c of a segment owns chunks c, c + SEG, ..
+    const int SEG = product_segment(RPU), RS = product_row_stride(CH, SEG);
+    const int my_row = lane / SEG, chunk = lane % SEG;
+    const bool row_active = my_row < RPU;
+    const int my_gate = row_active ? my_row / k_w : 0;
 
     // ---- shared memory carve-up ----
     uint4* sW = reinterpret_cast<uint4*>(smem_raw);                              // [PR][RS]
     uint4* sZ = sW + (size_t)PR * RS;                                            // [KA][CH]
-    int* sP = reinterpret_cast<int*>(sZ + KA * CH);                              // [PARTS][PR][KA]
-    float* sAlpha = reinterpret_cast<float*>(sP + PARTS * PR * KA);              // [PR]
+    float* sAlpha = reinterpret_cast<float*>(sZ + KA * CH);                      // [PR]
     float* sBias = sAlpha + PR;                                                  // [upc][4]
-    QuantScratch<KA>* scratch = reinterpret_cast<QuantScratch<KA>*>(
-        (reinterpret_cast<uintptr_t>(sBias + upc * 4) + 15) & ~uintptr_t(15));
+    float* sH = sBias + upc * 4;                                                 // [upc] h of the unit
+    float* sC = sH + upc;                                                        // [upc] c of the unit (LSTM)
+    QuantScratch<KA, NW>* scratch = reinterpret_cast<QuantScratch<KA, NW>*>(
+        (reinterpret_cast<uintptr_t>(sC + upc) + 15) & ~uintptr_t(15));
 
     // ---- resident weights: local plane-row pr = (ul * GATES + gate) * k_w + i ----
     {
@@ -128,81 +146,133 @@ rnn_persistent_kernel(PersistArgs a)
             const int ul = idx >> 2, s = idx & 3, u = u0 + ul;
             sBias[idx] = (a.bias && u < a.H) ? __ldg(a.bias + (size_t)s * a.H + u) : 0.0f;
         }
-    }
-
-    // epilogue role: thread e = ul * 4 + gate slot (slot 3 idle for the GRU), kept inside aligned quads
-    const int ep_ul = tid >> 2, ep_gate = tid & 3;
-    const int ep_warps = (upc * 4 + 31) >> 5;
-    const bool ep_valid = ep_ul < upc && ep_gate < GATES && (u0 + ep_ul) < a.H;
-    const bool ep_leader = ep_valid && ep_gate == 0;
-    float c_state = 0.0f, h_state = 0.0f;
-    if (ep_leader) {
-        h_state = __ldg(a.h0 + u0 + ep_ul);
-        if (!GRU) c_state = __ldg(a.c0 + u0 + ep_ul);
+        for (int ul = tid; ul < upc; ul += NT) {
+            const int u = u0 + ul;
+            sH[ul] = (u < a.H) ? __ldg(a.h0 + u) : 0.0f;
+            sC[ul] = (!GRU && u < a.H) ? __ldg(a.c0 + u) : 0.0f;
+        }
+        for (int q = tid; q < KA * wpr; q += NT) reinterpret_cast<uint32_t*>(sZ)[q] = 0u;   // plane words no thread owns
+        quant_scratch_init(*scratch);
     }
     __syncthreads();
 
+    // ---- element ownership: thread tid holds the EPT consecutive elements e0 .. e0 + EPT - 1 of z, so the sign bits
+    // the quantizer leaves in a register ARE a byte (half-word) of the packed plane ----
+    const int e0 = tid * EPT;
+    uint32_t valid = 0, hmask = 0;
+#pragma unroll
+    for (int j = 0; j < EPT; ++j) {
+        if (e0 + j < n) valid |= 1u << j;
+        if (e0 + j >= a.I && e0 + j < n) hmask |= 1u << j;
+    }
+    const bool vec = a.vec_ok != 0;                    // no thread straddles x and h, 16-byte loads are aligned
+    const int copies = a.copies;
+    const size_t hs = a.hx_stride;
+    const int my_copy = (int)(blockIdx.x % (unsigned)copies);
+    int parity = 0;
+
 #ifdef AMQ_PHASE_TIMING
-    long long ph[5] = {0, 0, 0, 0, 0};
+    long long ph[4] = {0, 0, 0, 0};
     long long tp = clock64();
 #endif
 
     for (int t = 0; t < a.steps; ++t) {
-        // ---- 1. gather z = [x_t ; h_{t-1}] (element j * NT + tid) ----
+        // ---- 1. gather z = [x_t ; h_{t-1}] ----
         float w[EPT];
-        uint32_t valid = 0, pending = 0;
-        const float* x = a.x_seq + (size_t)t * a.I;
-        const unsigned long long* hx = a.hx + (size_t)(t & 1) * a.H;
 #pragma unroll
-        for (int j = 0; j < EPT; ++j) {
-            const int e = j * NT + tid;
-            w[j] = 0.0f;
-            if (e < a.I) { w[j] = __ldg(x + e); valid |= 1u << j; }
-            else if (e < n) {
-                valid |= 1u << j;
-                if (t == 0) w[j] = __ldg(a.h0 + (e - a.I)); else pending |= 1u << j;
+        for (int j = 0; j < EPT; ++j) w[j] = 0.0f;
+        uint32_t pending = 0;
+        const float* x = a.x_seq + (size_t)t * a.I;
+        const unsigned long long* hx = a.hx + ((size_t)(t & 1) * copies + my_copy) * hs;
+        const unsigned want = (unsigned)t + a.tag_bias;
+        if (vec && e0 < a.I) {
+#pragma unroll
+            for (int q = 0; q < EPT / 4; ++q) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(x + e0) + q);
+                w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
             }
-        }
-        unsigned spins = 0;
-        while (pending) {
+        } else if (t == 0 || !vec) {
 #pragma unroll
             for (int j = 0; j < EPT; ++j) {
-                if ((pending >> j) & 1u) {
-                    const unsigned long long v = ld_relaxed_u64(hx + (j * NT + tid - a.I));
-                    if ((unsigned)(v >> 32) == (unsigned)t) {
-                        w[j] = __uint_as_float((unsigned)v);
-                        pending &= ~(1u << j);
+                const int e = e0 + j;
+                if (e < a.I) w[j] = __ldg(x + e);
+                else if (e < n) { if (t == 0) w[j] = __ldg(a.h0 + (e - a.I)); else pending |= 1u << j; }
+            }
+        } else {
+            pending = hmask;
+        }
+        unsigned spins = 0;
+        if (vec) {
+            // words come in aligned pairs (H is even and so is every thread's first index)
+            while (pending) {
+#pragma unroll
+                for (int q = 0; q < EPT / 2; ++q) {
+                    if ((pending >> (2 * q)) & 3u) {
+                        const ulonglong2 v = ld_relaxed_v2_u64(hx + (e0 - a.I) + 2 * q);
+                        if ((unsigned)(v.x >> 32) == want) { w[2 * q] = __uint_as_float((unsigned)v.x); pending &= ~(1u << (2 * q)); }
+                        if ((unsigned)(v.y >> 32) == want) { w[2 * q + 1] = __uint_as_float((unsigned)v.y); pending &= ~(2u << (2 * q)); }
                     }
                 }
+                if (++spins > a.poll_limit) break;
             }
-            if (++spins > POLL_LIMIT) break;
+        } else {
+            while (pending) {
+#pragma unroll
+                for (int j = 0; j < EPT; ++j) {
+                    if ((pending >> j) & 1u) {
+                        const unsigned long long v = ld_relaxed_u64(hx + (e0 + j - a.I));
+                        if ((unsigned)(v >> 32) == want) {
+                            w[j] = __uint_as_float((unsigned)v);
+                            pending &= ~(1u << j);
+                        }
+                    }
+                }
+                if (++spins > a.poll_limit) break;
+            }
         }
-        if (__syncthreads_or(pending != 0)) {          // some producer never arrived: give up, all together
+        int gave_up = pending != 0;                    // some producer never arrived
+        AMQ_PHASE(0);
+
+        // ---- 2. on-line quantization of z (Algorithm 2); its first barrier also takes the give-up vote ----
+        float beta[KA];
+        uint32_t bits[KA];
+        quantize_group<KA, EPT, NW>(w, valid, n, a.T, beta, bits, *scratch, &gave_up, &parity);
+        if (gave_up) {                                 // uniform over the CTA: leave together
             if (tid == 0) atomicExch(a.status, 1u);
             return;
         }
-        AMQ_PHASE(0);
-
-        // ---- 2. on-line quantization of z (Algorithm 2), planes packed into shared memory ----
-        float beta[KA];
-        uint32_t bits[KA];
-        quantize_group<KA, EPT, true>(w, valid, n, a.T, beta, bits, *scratch);
         AMQ_PHASE(1);
-        pack_group<KA, EPT>(bits, lane, warp, NT / 32, wpr, reinterpret_cast<uint32_t*>(sZ));
+        if (e0 < wpr * 32) {                           // this thread's bits lie inside the plane
+#pragma unroll
+            for (int i = 0; i < KA; ++i) {
+                if (EPT == 8) reinterpret_cast<uint8_t*>(sZ)[(size_t)i * wpr * 4 + tid] = (uint8_t)bits[i];
+                else reinterpret_cast<uint16_t*>(sZ)[(size_t)i * wpr * 2 + tid] = (uint16_t)bits[i];
+            }
+        }
         __syncthreads();
         AMQ_PHASE(2);
 
-        // ---- 3. binary product: P[pr][j] = popcount(W plane-row pr XOR z plane j) ----
-        for (int it = 0; it < pr_iters; ++it) {
-            const int pr = it * NSEG + seg;
+        // ---- 3. one warp per hidden unit: binary product, coefficients, gates, state update, publish ----
+        float beta_sum = 0.0f;
+#pragma unroll
+        for (int j = 0; j < KA; ++j) beta_sum += beta[j];
+        for (int ul = warp; ul < upc; ul += NW) {
+            const int u = u0 + ul;
+            if (u >= a.H) break;
             int acc[PARTS][KA];
 #pragma unroll
             for (int pt = 0; pt < PARTS; ++pt)
 #pragma unroll
                 for (int j = 0; j < KA; ++j) acc[pt][j] = 0;
-            if (pr < PR) {
+            const float al = row_active ? sAlpha[ul * RPU + my_row] : 0.0f;
+            const float* b4 = sBias + ul * 4;
+            const float bias_own = b4[my_gate];
+            const float state_old = GRU ? sH[ul] : sC[ul];
+            if (row_active) {
+                const uint4* wrow = sW + (size_t)(ul * RPU + my_row) * RS;
+#pragma unroll 4
                 for (int c = chunk; c < CH; c += SEG) {
-                    const uint4 wv = sW[(size_t)pr * RS + c];
+                    const uint4 wv = wrow[c];
                     const bool in_x = c * 128 < a.I;          // GRU only; the host requires I % 128 == 0
 #pragma unroll
                     for (int j = 0; j < KA; ++j) {
@@ -212,110 +282,107 @@ rnn_persistent_kernel(PersistArgs a)
                     }
                 }
             }
+            // this lane's share of its plane-row's dot products, weighted by the activation coefficients: the column
+            // count enters once per row (lane 0 of the segment); then the segment's lanes are added up
+            float yrow[PARTS];
+#pragma unroll
+            for (int pt = 0; pt < PARTS; ++pt) {
+                const int len = GRU ? (pt == 0 ? a.I : a.H) : n;
+                float s = (chunk == 0) ? (float)len * beta_sum : 0.0f;
+#pragma unroll
+                for (int j = 0; j < KA; ++j) s -= beta[j] * (float)(2 * acc[pt][j]);
+                yrow[pt] = al * s;
+            }
             for (int off = SEG >> 1; off > 0; off >>= 1) {
 #pragma unroll
-                for (int pt = 0; pt < PARTS; ++pt)
-#pragma unroll
-                    for (int j = 0; j < KA; ++j) acc[pt][j] += __shfl_xor_sync(0xffffffffu, acc[pt][j], off);
+                for (int pt = 0; pt < PARTS; ++pt) yrow[pt] += __shfl_xor_sync(0xffffffffu, yrow[pt], off);
             }
-            if (chunk == 0 && pr < PR) {
-#pragma unroll
-                for (int pt = 0; pt < PARTS; ++pt)
-#pragma unroll
-                    for (int j = 0; j < KA; ++j) sP[(pt * PR + pr) * KA + j] = acc[pt][j];
-            }
-        }
-        __syncthreads();
-        AMQ_PHASE(3);
-
-        // ---- 4. coefficients, gates, state update; the leader of each unit publishes h ----
-        if (warp < ep_warps) {
+            // the k_w planes of this lane's gate, added in plane order
             float y[PARTS];
 #pragma unroll
             for (int pt = 0; pt < PARTS; ++pt) y[pt] = 0.0f;
-            if (ep_valid) {
-                const int lr = ep_ul * GATES + ep_gate;
+            for (int i = 0; i < k_w; ++i) {
+                const int src = (my_gate * k_w + i) * SEG;
 #pragma unroll
-                for (int pt = 0; pt < PARTS; ++pt) {
-                    const int len = GRU ? (pt == 0 ? a.I : a.H) : n;
-                    for (int i = 0; i < k_w; ++i) {
-                        const float al = sAlpha[lr * k_w + i];
-#pragma unroll
-                        for (int j = 0; j < KA; ++j)
-                            y[pt] += al * beta[j] * (float)(len - 2 * sP[(pt * PR + lr * k_w + i) * KA + j]);
-                    }
-                }
+                for (int pt = 0; pt < PARTS; ++pt) y[pt] += __shfl_sync(0xffffffffu, yrow[pt], src);
             }
-            const int quad = lane & ~3;
-            float h_new;
+            const int gate_stride = k_w * SEG;             // first lane of gate g: g * gate_stride
+            float h_new, c_new = 0.0f;
             if (!GRU) {
-                const float pre = y[0] + sBias[(ep_ul < upc ? ep_ul : 0) * 4 + ep_gate];
-                const float act = (ep_gate == 3) ? fast_tanh(pre) : logistic(pre);
-                const float ig = __shfl_sync(0xffffffffu, act, quad + 0);
-                const float fg = __shfl_sync(0xffffffffu, act, quad + 1);
-                const float og = __shfl_sync(0xffffffffu, act, quad + 2);
-                const float gg = __shfl_sync(0xffffffffu, act, quad + 3);
-                c_state = fg * c_state + ig * gg;
-                h_new = og * fast_tanh(c_state);
+                // logistic for i, f, o; tanh(v) = 2 logistic(2 v) - 1 for g: one exponential either way
+                const float sc = (my_gate == 3) ? 2.0f : 1.0f;
+                const float act = sc * logistic(sc * (y[0] + bias_own)) - (sc - 1.0f);
+                const float ig = __shfl_sync(0xffffffffu, act, 0);
+                const float fg = __shfl_sync(0xffffffffu, act, gate_stride);
+                const float og = __shfl_sync(0xffffffffu, act, 2 * gate_stride);
+                const float gg = __shfl_sync(0xffffffffu, act, 3 * gate_stride);
+                c_new = fg * state_old + ig * gg;
+                h_new = og * fast_tanh(c_new);
             } else {
-                const float* b4 = sBias + (ep_ul < upc ? ep_ul : 0) * 4;
                 const float yx = y[0], yh = y[PARTS - 1];
-                const float gate_rz = logistic(yx + yh + b4[ep_gate & 1]);        // meaningful for slots 0, 1
-                const float rg = __shfl_sync(0xffffffffu, gate_rz, quad + 0);
-                const float zg = __shfl_sync(0xffffffffu, gate_rz, quad + 1);
-                const float cand_own = fast_tanh(yx + b4[2] + rg * (yh + b4[3]));  // meaningful for slot 2
-                const float cand = __shfl_sync(0xffffffffu, cand_own, quad + 2);
-                h_new = (1.0f - zg) * cand + zg * h_state;
+                const float gate_rz = logistic(yx + yh + b4[my_gate & 1]);        // meaningful for gates 0, 1
+                const float rg = __shfl_sync(0xffffffffu, gate_rz, 0);
+                const float zg = __shfl_sync(0xffffffffu, gate_rz, gate_stride);
+                const float cand_own = fast_tanh(yx + b4[2] + rg * (yh + b4[3]));  // meaningful for gate 2
+                const float cand = __shfl_sync(0xffffffffu, cand_own, 2 * gate_stride);
+                h_new = (1.0f - zg) * cand + zg * state_old;
             }
-            if (ep_leader) {
-                h_state = h_new;
-                const int u = u0 + ep_ul;
+            // every lane holds the unit's new state; lane r < copies publishes copy r
+            if (lane < copies) {
                 const unsigned long long word =
                     ((unsigned long long)(unsigned)(t + 1) << 32) | (unsigned long long)__float_as_uint(h_new);
-                st_relaxed_u64(a.hx + (size_t)((t + 1) & 1) * a.H + u, word);
+                st_relaxed_u64(a.hx + ((size_t)((t + 1) & 1) * copies + lane) * hs + u, word);
+            }
+            __syncwarp();                                  // all lanes have read the old state
+            if (lane == 0) {
+                sH[ul] = h_new;
+                if (!GRU) sC[ul] = c_new;
                 if (a.h_seq) a.h_seq[(size_t)t * a.H + u] = h_new;
             }
         }
-        AMQ_PHASE(4);
+        AMQ_PHASE(3);
     }
 #ifdef AMQ_PHASE_TIMING
     if (tid == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {
-        for (int i = 0; i < 5; ++i)
+        for (int i = 0; i < 4; ++i)
             a.status[8 + (blockIdx.x ? 8 : 0) + i] = (uint32_t)(ph[i] / (a.steps > 0 ? a.steps : 1));
     }
 #endif
 
-    if (ep_leader) {
-        a.h_last[u0 + ep_ul] = h_state;
-        if (!GRU) a.c_last[u0 + ep_ul] = c_state;
+    __syncthreads();
+    for (int ul = tid; ul < upc; ul += NT) {
+        const int u = u0 + ul;
+        if (u < a.H) {
+            a.h_last[u] = sH[ul];
+            if (!GRU) a.c_last[u] = sC[ul];
+        }
     }
 }
 
-size_t persistent_smem_bytes(int upc, int gates, int k_w, int k_a, int wpr)
+template <int NW>
+size_t persistent_smem_bytes(int upc, int gates, int k_w, int wpr)
 {
     const size_t PR = (size_t)upc * gates * k_w, CH = wpr / 4;
-    const size_t RS = product_row_stride((int)CH, product_segment((int)PR, (int)CH));
-    size_t b = PR * RS * 16 + (size_t)k_a * CH * 16 + (gates == 3 ? 2 : 1) * PR * k_a * 4 + PR * 4 + (size_t)upc * 16;
-    return b + 16 + sizeof(QuantScratch<AMQ_MAX_K>);       // alignment slack + quantizer scratch
+    const size_t RS = product_row_stride((int)CH, product_segment(gates * k_w));
+    const size_t b = PR * RS * 16 + (size_t)AMQ_MAX_K * CH * 16 + PR * 4 + (size_t)upc * 16 + (size_t)upc * 8;
+    return b + 16 + sizeof(QuantScratch<AMQ_MAX_K, NW>);   // alignment slack + quantizer scratch
 }
 
 int device_sm_count()
 {
-    static thread_local int cached_dev = -1, cached_sms = 0;
-    int dev = 0;
+    int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (dev != cached_dev) {
-        int sms = 0;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        cached_dev = dev; cached_sms = sms;
-    }
-    return cached_sms;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return sms;
 }
 
-template <int KA, int EPT, bool GRU>
+constexpr int NT_SMALL = 128;            // threads per CTA for vectors of up to 1024 elements (8 per thread)
+constexpr int NT_LARGE = 256;            // up to 2048 (8 per thread) and 4096 (16 per thread)
+
+template <int KA, int EPT, bool GRU, int NT>
 amq_status launch(const PersistArgs& a, int grid, size_t smem, cudaStream_t st)
 {
-    auto kernel = rnn_persistent_kernel<KA, EPT, GRU>;
+    auto kernel = rnn_persistent_kernel<KA, EPT, GRU, NT>;
     AMQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     PersistArgs args = a;
     void* params[] = {&args};
@@ -333,8 +400,12 @@ amq_status launch(const PersistArgs& a, int grid, size_t smem, cudaStream_t st)
 template <int KA, bool GRU>
 amq_status launch_ept(const PersistArgs& a, int n, int grid, size_t smem, cudaStream_t st)
 {
-    if (n <= NT * 4) return launch<KA, 4, GRU>(a, grid, smem, st);
-    return launch<KA, 8, GRU>(a, grid, smem, st);
+    PersistArgs b = a;
+    const int ept = n <= NT_LARGE * 8 ? 8 : 16;
+    b.vec_ok = (a.I % ept) == 0 && (a.H % 2) == 0 && (reinterpret_cast<uintptr_t>(a.x_seq) & 15u) == 0;
+    if (n <= NT_SMALL * 8) return launch<KA, 8, GRU, NT_SMALL>(b, grid, smem, st);
+    if (n <= NT_LARGE * 8) return launch<KA, 8, GRU, NT_LARGE>(b, grid, smem, st);
+    return launch<KA, 16, GRU, NT_LARGE>(b, grid, smem, st);
 }
 
 }  // namespace
@@ -343,16 +414,15 @@ bool persistent_supported(int I, int H, int batch, int k_w, int k_a, bool gru, i
                           size_t* smem_out)
 {
     const int n = I + H;
-    if (batch != 1 || n > NT * 8) return false;
+    if (batch != 1 || n > NT_LARGE * 16) return false;
     if (gru && (I % 128) != 0) return false;
     const int sms = device_sm_count();
     if (sms <= 0) return false;
     const int wpr = words_per_row(n);
-    if (wpr / 4 > 32) return false;
     const int upc = (H + sms - 1) / sms;
-    if (upc * 4 > NT) return false;
     const int grid = (H + upc - 1) / upc;
-    const size_t smem = persistent_smem_bytes(upc, gru ? 3 : 4, k_w, k_a, wpr);
+    const size_t smem = persistent_smem_bytes<NT_LARGE / 32>(upc, gru ? 3 : 4, k_w, wpr);
+    (void)k_a;
     if (smem > 200 * 1024) return false;
     *grid_out = grid; *upc_out = upc; *smem_out = smem;
     return true;
@@ -362,13 +432,15 @@ amq_status launch_rnn_persistent(const uint32_t* Wcodes, const float* Walpha, co
                                  int I, int H, int k_w, int k_a, int T, bool gru,
                                  const float* x_seq, int steps, const float* h0, const float* c0,
                                  float* h_seq, float* h_last, float* c_last,
-                                 unsigned long long* hx, uint32_t* status, cudaStream_t st)
+                                 unsigned long long* hx, uint32_t* status, cudaStream_t st,
+                                 unsigned poll_limit, unsigned tag_bias)
 {
     int grid = 0, upc = 0;
     size_t smem = 0;
     if (!persistent_supported(I, H, 1, k_w, k_a, gru, &grid, &upc, &smem)) return AMQ_ERR_UNSUPPORTED;
-    PersistArgs a{Wcodes, Walpha, bias, I, H, k_w, T, steps, x_seq, h0, c0, h_seq, h_last, c_last, hx, status,
-                  upc, words_per_row(I + H)};
+    PersistArgs a{Wcodes, Walpha, bias, I, H, k_w, T, steps, x_seq, h0, c0, h_seq, h_last, c_last, hx,
+                  persistent_exchange_stride(H), 0, status,
+                  upc, words_per_row(I + H), PERSISTENT_EXCHANGE_COPIES, poll_limit ? poll_limit : POLL_LIMIT, tag_bias};
     const int n = I + H;
     if (gru) {
         switch (k_a) {
