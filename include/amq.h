@@ -81,8 +81,9 @@ AMQ_API size_t amq_codes_bytes(int rows, int n, int k);
  * Readings where the paper is silent: sign(0) = +1; the level table is sorted by (value, code index)
  * with plane 0 the most significant code bit; a refit whose k x k system has a pivot below 1e-9 * n
  * (Gaussian elimination with partial pivoting, in double) is skipped and keeps the previous coefficients.
- * Sums over a row are accumulated in fp32 per thread and in fp64 across threads; the solve is fp64;
- * levels, thresholds and comparisons are fp32.
+ * Sums over a row are accumulated in fp32 (per thread, then across threads in a fixed order, so results repeat
+ * bit for bit); B^T B is exact integer arithmetic; the k x k solve is fp64 for k >= 3 and error-compensated fp32 for
+ * k = 2; levels, thresholds and comparisons are fp32.
  */
 AMQ_API amq_status amq_quantize(const float* x, int rows, int n, int ldx, int k, int T,
                         uint32_t* codes, float* coeffs, void* stream);
@@ -200,8 +201,8 @@ AMQ_API amq_status amq_gru_step(const uint32_t* Wcodes, const float* Walpha, con
                         void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * `steps` consecutive steps without returning to the host ("RNNs can only be executed sequentially",
- * Sec. 1: step t+1 consumes h_t).  x_seq [steps][batch][I]; h0, c0 [batch][H];
+ * `steps` consecutive steps without returning to the host (step t+1 consumes h_t, so a sequence is one
+ * dependency chain: Sec. 1).  x_seq [steps][batch][I]; h0, c0 [batch][H];
  * h_seq [steps][batch][H] out or NULL; h_last, c_last [batch][H] out.  Outputs must not alias inputs.
  */
 AMQ_API amq_status amq_lstm_sequence(const uint32_t* Wcodes, const float* Walpha, const float* bias,
@@ -327,6 +328,22 @@ AMQ_API amq_status amq_gru_sequence_host(const uint32_t* Wcodes, const float* Wa
                                  float* h_seq_host, float* h_last_host,
                                  void* workspace, size_t workspace_bytes,
                                  void* staging, size_t staging_bytes, void* stream);
+
+/*
+ * Test aid for the give-up path of the batch-1 sequence kernel (the paper has no counterpart).  Same arguments as
+ * amq_lstm_sequence with batch = 1 and steps >= 2, plus `poll_limit` (1 .. 65536): the kernel runs with that many
+ * polls as the limit of every wait for the other CTAs' h values and expects step tags that no CTA ever publishes.
+ * Step 0 (which waits for nothing) runs normally; in step 1 every wait runs out, every CTA records the failure in
+ * the workspace status word and returns, and the outputs are left unwritten.  The call returns AMQ_OK when the launch
+ * was enqueued; amq_workspace_status then returns AMQ_ERR_TIMEOUT, and the next cell call on the workspace clears it.
+ * Nothing faults or hangs: the waits are the ordinary bounded ones with a smaller bound.  AMQ_ERR_UNSUPPORTED when the
+ * problem is not one the batch-1 sequence kernel takes.
+ */
+AMQ_API amq_status amq_selftest_sequence_give_up(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                                         int I, int H, int k_w,
+                                         const float* x_seq, int steps, const float* h0, const float* c0,
+                                         int k_a, int T, float* h_last, float* c_last,
+                                         void* workspace, size_t workspace_bytes, unsigned poll_limit, void* stream);
 
 /*
  * Synchronises `stream`, then reads the status word at the start of a cell workspace: AMQ_OK, or

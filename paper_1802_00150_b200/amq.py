@@ -52,6 +52,8 @@ EXPORTS = {
     "amq_gru_sequence_host": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _int, _vp, _int, _int, _int,
                                      _vp, _vp, _vp, _sz, _vp, _sz, _vp]),
     "amq_workspace_status": (_int, [_vp, _vp]),
+    "amq_selftest_sequence_give_up": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _int, _vp, _vp, _int, _int,
+                                             _vp, _vp, _vp, _sz, ctypes.c_uint, _vp]),
     "amq_gru_original_workspace_bytes": (_sz, [_int, _int, _int, _int]),
     "amq_gru_step_original": (_int, [_vp, _vp, _vp, _int, _int, _int, _vp, _vp, _int, _int, _int, _vp, _vp, _sz, _vp]),
     "amq_quantize_variant": (_int, [_vp, _int, _int, _int, _int, _int, _int, _int, _vp, _vp, _vp]),
@@ -251,6 +253,18 @@ def lstm_sequence(Wcodes, Walpha, bias, I, H, x_seq, h0, c0, k_a, T, workspace, 
                                   _ptr(c0), batch, k_a, T, _ptr(h_seq), _ptr(h_last), _ptr(c_last),
                                   _ptr(workspace), workspace.numel(), _stream()))
     return h_seq, h_last, c_last
+
+
+def selftest_sequence_give_up(Wcodes, Walpha, bias, I, H, x_seq, h0, c0, k_a, T, workspace, poll_limit):
+    """Test aid: the batch-1 LSTM sequence kernel with waits that run out (see amq.h).  Returns (h_last, c_last),
+    which the kernel leaves unwritten; read the outcome with workspace_status."""
+    Wcodes, Walpha = _dev(Wcodes, torch.int32, "Wcodes"), _dev(Walpha, torch.float32, "Walpha")
+    x_seq, h0, c0 = _dev(x_seq, torch.float32, "x_seq"), _dev(h0, torch.float32, "h0"), _dev(c0, torch.float32, "c0")
+    h_last, c_last = torch.zeros_like(h0), torch.zeros_like(c0)
+    _check(_lib.amq_selftest_sequence_give_up(_ptr(Wcodes), _ptr(Walpha), _ptr(bias), I, H, Wcodes.shape[1], _ptr(x_seq),
+                                              x_seq.shape[0], _ptr(h0), _ptr(c0), k_a, T, _ptr(h_last), _ptr(c_last),
+                                              _ptr(workspace), workspace.numel(), poll_limit, _stream()))
+    return h_last, c_last
 
 
 def gru_sequence(Wcodes, Walpha, bias, I, H, x_seq, h0, k_a, T, workspace, want_h_seq=False,

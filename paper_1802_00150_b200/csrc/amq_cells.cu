@@ -32,12 +32,12 @@ bool use_persistent(const CellCall& c)
 
 amq_status enqueue_persistent(const CellCall& c, const CellWorkspace& ws, const float* x_seq, int steps,
                               const float* h0, const float* c0, float* h_seq, float* h_last, float* c_last,
-                              cudaStream_t st)
+                              cudaStream_t st, unsigned poll_limit = 0, unsigned tag_bias = 0)
 {
     // the caller has cleared the status words and, for more than one step, the exchange words behind them (stale
     // step tags must not match; a single step polls nothing)
     return launch_rnn_persistent(c.Wcodes, c.Walpha, c.bias, c.I, c.H, c.k_w, c.k_a, c.T, c.gru, x_seq, steps,
-                                 h0, c0, h_seq, h_last, c_last, ws.hx, ws.status, st);
+                                 h0, c0, h_seq, h_last, c_last, ws.hx, ws.status, st, poll_limit, tag_bias);
 }
 
 // (inputs come from the preceding kernels of the stream: ordinary loads after the wait, no read-only path)
@@ -261,6 +261,26 @@ amq_status amq_gru_sequence_host(const uint32_t* Wcodes, const float* Walpha, co
     amq::CellCall c{Wcodes, Walpha, bias, I, H, k_w, batch, k_a, T, true};
     return amq::sequence_host_entry(c, x_seq_host, steps, h0_host, nullptr, h_seq_host, h_last_host, nullptr,
                                     workspace, workspace_bytes, staging, staging_bytes, (cudaStream_t)stream);
+}
+
+amq_status amq_selftest_sequence_give_up(const uint32_t* Wcodes, const float* Walpha, const float* bias,
+                                         int I, int H, int k_w,
+                                         const float* x_seq, int steps, const float* h0, const float* c0,
+                                         int k_a, int T, float* h_last, float* c_last,
+                                         void* workspace, size_t workspace_bytes, unsigned poll_limit, void* stream)
+{
+    amq::CellCall c{Wcodes, Walpha, bias, I, H, k_w, 1, k_a, T, false};
+    amq_status s = amq::validate(c, workspace, workspace_bytes);
+    if (s != AMQ_OK) return s;
+    if (steps < 2 || !h0 || !c0 || !h_last || !c_last || (I > 0 && !x_seq) || h_last == h0 || c_last == c0)
+        return AMQ_ERR_INVALID_ARG;
+    if (poll_limit < 1 || poll_limit > 65536) return AMQ_ERR_INVALID_ARG;
+    if (!amq::use_persistent(c)) return AMQ_ERR_UNSUPPORTED;
+    amq::CellWorkspace ws = amq::carve_cell_workspace(workspace, I, H, 1, k_a);
+    AMQ_CUDA_TRY(cudaMemsetAsync(ws.status, 0, 256 + ws.hx_bytes, (cudaStream_t)stream));
+    // expected tags are offset by 2^30: the tags the CTAs publish (1 .. steps) never match
+    return amq::enqueue_persistent(c, ws, x_seq, steps, h0, c0, nullptr, h_last, c_last, (cudaStream_t)stream,
+                                   poll_limit, 1u << 30);
 }
 
 amq_status amq_workspace_status(const void* workspace, void* stream)

@@ -146,3 +146,27 @@ def test_argument_validation_of_the_widened_entry_points(lib):
     lib.amq_lstm_paper_workspace_bytes.argtypes = [ci] * 4
     assert lib.amq_lstm_paper_workspace_bytes(8, 2, 3, 2) > lib.amq_lstm_paper_workspace_bytes(8, 2, 1, 2) > 0
     assert lib.amq_lstm_paper_workspace_bytes(8, 2, 3, 0) == 0
+
+
+def test_argument_validation_of_the_give_up_selftest(lib):
+    """The test aid for the give-up path is validated on the host like every other entry (no launch below)."""
+    vp, ci, sz, cu = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_uint
+    fake, fake2, fake3 = vp(0x1000), vp(0x2000), vp(0x3000)
+    lib.amq_cell_workspace_bytes.restype = sz
+    lib.amq_cell_workspace_bytes.argtypes = [ci] * 4
+    need = lib.amq_cell_workspace_bytes(8, 8, 1, 2)
+    st = lib.amq_selftest_sequence_give_up
+    st.argtypes = [vp, vp, vp, ci, ci, ci, vp, ci, vp, vp, ci, ci, vp, vp, vp, sz, cu, vp]
+    ok_args = [fake, fake, None, 8, 8, 2, fake, 3, fake, fake, 2, 2, fake2, fake3, fake, need, 100, None]
+    bad = list(ok_args); bad[15] = need - 1
+    assert st(*bad) == -4                                                  # workspace too small
+    bad = list(ok_args); bad[7] = 1
+    assert st(*bad) == -1                                                  # one step waits for nothing
+    bad = list(ok_args); bad[16] = 0
+    assert st(*bad) == -1                                                  # poll limit out of range
+    bad = list(ok_args); bad[16] = 1 << 17
+    assert st(*bad) == -1
+    bad = list(ok_args); bad[12] = fake
+    assert st(*bad) == -1                                                  # h_last == h0
+    bad = list(ok_args); bad[10] = 5
+    assert st(*bad) == -2                                                  # bits

@@ -81,9 +81,67 @@ def test_lstm1024_batch1_sequence_workload(amq):
     # the first step of the free-running sequence starts from the same state as the oracle
     _, beta = oracle.quantize_rows(np.concatenate([xs[0].astype(np.float64), states[0][0]], axis=1), wl.k_a, wl.T)
     assert np.abs(g_seq[0].cpu().numpy() - states[1][0]).max() <= state_tolerance(Wa, beta, wl.n)
+    # the 35-step launch (all CTAs exchanging h) equals 35 chained single-step launches bit for bit, so the
+    # teacher-forced parity of the step above carries over to every step of the sequence launch
+    h, c = dev(h0), dev(c0)
+    for s in range(wl.steps):
+        h, c = amq.lstm_step(Wcodes, Walpha, None, wl.I, wl.H, dev(xs[s]), h, c, wl.k_a, wl.T, ws)
+        assert torch.equal(h, g_seq[s]), s
+    assert torch.equal(c, g_c)
+    # five more runs of the sequence launch: the exchange must not make results depend on timing
+    for _ in range(5):
+        r_seq, _, r_c = amq.lstm_sequence(Wcodes, Walpha, None, wl.I, wl.H, dev(xs), dev(h0), dev(c0), wl.k_a, wl.T, ws,
+                                          want_h_seq=True)
+        assert torch.equal(r_seq, g_seq) and torch.equal(r_c, g_c)
     drift = max(np.abs(g_seq[s].cpu().numpy() - states[s + 1][0]).max() for s in range(wl.steps))
     print("free-running max |dh| over 35 steps: %.3g" % drift)
-    assert np.isfinite(drift) and drift <= 0.5
+    assert np.isfinite(drift)
+
+
+@pytest.mark.parametrize("name", ["lstm1024_b64", "gru2048_b256"])
+def test_batched_sequence_workloads(amq, name):
+    """The 35-step batched sequences bench.py times: the sequence call equals the chained step calls bit for bit, and
+    sampled steps of sampled sequences, restarted from the library's own state, land on the oracle's next state."""
+    wl = synth.WORKLOADS[name]
+    _, Wcodes, Walpha, Wc, Wa = quantized_model(amq, wl)
+    ins = synth.inputs(wl)
+    xs, h0 = ins["x_seq"], ins["h0"]
+    c0 = ins.get("c0")
+    lstm = wl.cell == "lstm"
+    ws = amq.new_workspace(wl.I, wl.H, wl.batch, wl.k_a)
+    if lstm:
+        g_seq, g_last, g_c = amq.lstm_sequence(Wcodes, Walpha, None, wl.I, wl.H, dev(xs), dev(h0), dev(c0), wl.k_a, wl.T,
+                                               ws, want_h_seq=True)
+    else:
+        g_seq, g_last = amq.gru_sequence(Wcodes, Walpha, None, wl.I, wl.H, dev(xs), dev(h0), wl.k_a, wl.T, ws,
+                                         want_h_seq=True)
+    assert amq.workspace_status(ws) == 0 and amq.device_status() == 0
+    assert torch.equal(g_seq[-1], g_last)
+    sample_steps = (0, 1, 16, 34)
+    sample_seqs = (0, wl.batch // 2 + 1)
+    h, c = dev(h0), (dev(c0) if lstm else None)
+    for s in range(wl.steps):
+        h_prev, c_prev = h, c
+        if lstm:
+            h, c = amq.lstm_step(Wcodes, Walpha, None, wl.I, wl.H, dev(xs[s]), h_prev, c_prev, wl.k_a, wl.T, ws)
+        else:
+            h = amq.gru_step(Wcodes, Walpha, None, wl.I, wl.H, dev(xs[s]), h_prev, wl.k_a, wl.T, ws)
+        assert torch.equal(h, g_seq[s]), s
+        if s in sample_steps:
+            for b in sample_seqs:
+                xb = xs[s][b:b + 1]
+                hp = h_prev[b:b + 1].cpu().numpy()
+                _, beta = oracle.quantize_rows(np.concatenate([xb, hp], axis=1).astype(np.float64), wl.k_a, wl.T)
+                tol = state_tolerance(Wa, beta, wl.n)
+                if lstm:
+                    cp = c_prev[b:b + 1].cpu().numpy()
+                    h_ref, c_ref = oracle.lstm_step(Wc, Wa, None, wl.I, wl.H, xb, hp, cp, wl.k_a, wl.T)
+                    assert np.abs(c[b:b + 1].cpu().numpy() - c_ref).max() <= tol, (s, b)
+                else:
+                    h_ref = oracle.gru_step(Wc, Wa, None, wl.I, wl.H, xb, hp, wl.k_a, wl.T)
+                assert np.abs(h[b:b + 1].cpu().numpy() - h_ref).max() <= tol, (s, b)
+    if lstm:
+        assert torch.equal(c, g_c)
 
 
 @pytest.mark.parametrize("name", ["lstm1024_b64", "gru2048_b256"])

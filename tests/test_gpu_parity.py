@@ -99,13 +99,18 @@ def test_quantize_degenerate_rows(amq):
         assert parity.pad_bits_zero(c, n)
         assert np.all(parity.unpack_rows(c, n)[0] == 1) and np.all(coeffs.cpu().numpy()[0] == 0)
         assert np.all(parity.unpack_rows(c, n)[5] == 1)
+        # rows whose answer is known in closed form come back exactly (to fp32 rounding): an all-zero row, a constant
+        # row (one level carries everything), a row of one magnitude (alpha_1 = 0.5, the other planes idle)
+        for r in (0, 1, 2, 5):
+            assert np.abs(xhat[r] - x[r].astype(np.float64)).max() <= 1e-6 * np.abs(x[r]).max(), (k, r)
         for r in range(8):
             o_alpha, o_b = oracle.quantize(x[r].astype(np.float64), k, 2)
             rec = oracle.reconstruct(o_alpha, o_b)
             scale = np.abs(o_alpha).sum() + 1e-30
-            # compare reconstructions (several codes are correct when levels coincide)
+            # compare reconstructions (several codes are correct when levels coincide): duplicated values and exact
+            # ties may legitimately flip single elements on a decision boundary, counted as in the staged protocol
             mism = np.abs(rec - xhat[r]) > 2e-4 * scale
-            assert mism.mean() <= 0.01, (k, r, mism.sum())
+            assert mism.sum() <= (0 if r in (0, 1, 2, 5) else 3), (k, r, mism.sum())
 
 
 def test_quantize_strided_rows_and_reuse_of_outputs(amq):
@@ -367,7 +372,7 @@ def test_quantizer_variants_match_oracle(amq, rows, n, k, dist, method, final_re
     for r in range(rows):
         w = x[r].astype(np.float64)
         if np.array_equal(gb[r], ob[r]):
-            assert np.abs(g_coeffs[r] - o_coeffs[r]).max() <= parity.COEFF_REL * np.abs(o_coeffs[r]).max() + 1e-30, r
+            assert np.all(np.abs(g_coeffs[r] - o_coeffs[r]) <= parity.coefficient_bound(o_coeffs[r])), r
         else:
             differing += 1
             og, oo = oracle.objective(w, g_coeffs[r], gb[r]), oracle.objective(w, o_coeffs[r], ob[r])

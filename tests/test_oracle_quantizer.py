@@ -362,6 +362,45 @@ def test_variants_final_refit_and_refined_greedy():
         assert np.array_equal(codes[r], oracle.pack_planes(b))
 
 
+def test_refined_greedy_takes_its_later_bits_from_the_refitted_residue():
+    """Hand-worked vector on which the refit after the second bit changes the sign of two residues, so the third
+    bit of the refined method (Sec. 2: after every greedy bit ALL coefficients so far are re-solved, and the next
+    bit is taken from the residue those refitted coefficients leave) differs from plain greedy's third bit.
+
+    w = (-8, -6, -1, 0, 0), n = 5, sign(0) = +1.
+      bit 1: b1 = (-,-,-,+,+), alpha1 = (8+6+1)/5 = 3; the one-coefficient refit b1.w / n = 15/5 = 3 changes nothing.
+             residue w - 3 b1 = (-5, -3, 2, -3, -3).
+      bit 2: b2 = (-,-,+,-,-), alpha2 = (5+3+2+3+3)/5 = 3.2.
+             refit: b1.b2 = 1+1-1-1-1 = -1, b1.w = 15, b2.w = 8+6-1 = 13;  [[5,-1],[-1,5]] a = (15, 13)
+             -> a = ((5*15+13)/24, (5*13+15)/24) = (11/3, 10/3).
+             refined residue w - 11/3 b1 - 10/3 b2 = (-1, 1, -2/3, -1/3, -1/3)   -> b3 = (-,+,-,-,-)
+             greedy  residue w - 3 b1 - 3.2 b2     = (-1.8, 0.2, -1.2, 0.2, 0.2) -> b3 = (-,+,-,+,+)
+    The last coefficients are the least-squares fit to the three hand-derived planes (numpy, independent routine)."""
+    w = np.array([-8.0, -6.0, -1.0, 0.0, 0.0])
+    b1 = np.array([-1, -1, -1, 1, 1])
+    b2 = np.array([-1, -1, 1, -1, -1])
+    b3_refined = np.array([-1, 1, -1, -1, -1])
+    b3_greedy = np.array([-1, 1, -1, 1, 1])
+    # two bits: the refitted coefficients printed above
+    a2, c2 = oracle.refined_greedy(w, 2)
+    assert np.array_equal(c2, np.stack([b1, b2]))
+    assert np.allclose(a2, [11.0 / 3.0, 10.0 / 3.0], rtol=1e-14)
+    # three bits
+    a3, c3 = oracle.refined_greedy(w, 3)
+    assert np.array_equal(c3, np.stack([b1, b2, b3_refined]))
+    B = np.stack([b1, b2, b3_refined]).T.astype(np.float64)
+    assert np.allclose(a3, np.linalg.lstsq(B, w, rcond=None)[0], rtol=1e-12)
+    # plain greedy on the same vector keeps the unrefitted coefficients and lands on the other third plane
+    ag, cg = oracle.greedy(w, 3)
+    assert np.array_equal(cg, np.stack([b1, b2, b3_greedy]))
+    assert np.allclose(ag[:2], [3.0, 3.2], rtol=1e-14)
+    # and the refined result is the better fit, as the comparison of Tables 1-2 has it
+    assert oracle.objective(w, a3, c3) < oracle.objective(w, ag, cg)
+    # the variant entry point takes the same path
+    av, cv = oracle.quantize_variant(w, 3, 0, oracle.METHOD_REFINED_GREEDY, False)
+    assert np.array_equal(cv, c3) and np.array_equal(av, a3)
+
+
 def test_error_levels_of_the_methods_are_those_of_table_1_on_gaussian_rows():
     """Table 1 prints the relative MSE of greedy, refined and alternating quantization of trained LSTM weights.  Those
     weights are not available; rows of Gaussian noise are close to them in shape, and the oracle must then land near the
