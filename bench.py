@@ -32,8 +32,11 @@ METRIC = "quantized LSTM/GRU timesteps per second (timesteps x concurrent sequen
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by workload; the summaries are under profiles/.  None = not captured.
-NCU_TRAFFIC_BYTES = {"lstm1024_b1": 2331648 + 10496}     # rnn_persistent_kernel, profiles/rnn_persistent_kernel_lstm1024_b1.txt
+# dram__bytes_write.sum), keyed by workload; the summaries are under profiles/.  None = not captured for the
+# kernel as it stands.
+NCU_TRAFFIC_BYTES = {}
+# the same for the cold matrix-vector kernel on 131072 x 8192 at 2/2 bits (profiles/bgemv_kernel_131072x8192_k2k2.txt)
+NCU_TRAFFIC_GEMV_COLD_BYTES = 269500000
 
 
 def parse_args():
@@ -176,7 +179,7 @@ class ClockSampler:
                 self.samples.append((sm, [k for k, bit in names.items() if mask & bit]))
             except Exception:
                 pass
-            time.sleep(0.02)
+            time.sleep(0.004)
 
     def start(self):
         try:
@@ -213,7 +216,7 @@ class ClockSampler:
             sm = [s for s, _ in self.samples]
             reasons = sorted({r for _, rs in self.samples for r in rs})
             return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": float(self.max_sm),
-                    "reasons": reasons, "samples": len(sm), "source": "nvml, 20 ms period, during the timed region"}
+                    "reasons": reasons, "samples": len(sm), "source": "nvml, ~5 ms period, during the timed regions (device-resident steps and end-to-end steps)"}
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -365,9 +368,9 @@ def run_ours(args, wl):
     if rank == 0:
         sampler.start()
     ms, launches = timed(step, args.steps, max(args.warmup, 3))
-    clocks = sampler.stop() if rank == 0 else None
     total_ms = float(sum(ms))
     ms_e2e, _ = timed(step_e2e, max(3, min(args.steps, 20)), 3)
+    clocks = sampler.stop() if rank == 0 else None
     e2e_total_ms = float(sum(ms_e2e))
     e2e_iters = len(ms_e2e)
     if dist is not None:
@@ -393,7 +396,8 @@ def run_ours(args, wl):
         achieved = alg_bytes / (step_ms * 1e-3) / 1e9
         line = {
             "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "ms_per_step_median": float(np.median(ms)),
+            "ms_per_step_min": float(np.min(ms)), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "u32 popcount + f32", "data": "synthetic",
             "config": workload_config(wl, "flushed before every step by an untimed 256 MiB write; inside a step "
                                           "the packed weights are re-read from L2 by design"),
@@ -409,6 +413,11 @@ def run_ours(args, wl):
         }
         if not args.no_extras and world == 1:
             line["gemv_cold"] = cold_gemv(amq, torch, dev, flush, peak, peak_kind)
+            # the second half of the metric (binary matrix-vector product against the HBM peak) beside the first
+            first = line["gemv_cold"][0]
+            line["roofline"]["gemv_cold"] = {k: first[k] for k in ("workload", "ms", "ms_min", "achieved", "unit", "peak", "frac",
+                                                                   "peak_kind", "frac_of_nominal_8000", "algorithmic_bytes")}
+            line["roofline"]["gemv_cold"]["traffic"] = NCU_TRAFFIC_GEMV_COLD_BYTES
             line["gemv_rotated"] = rotated_gemv(amq, torch, dev, peak, peak_kind)
             line["batched"] = batched_lines(amq, torch, dev, flush, peak, peak_kind)
             assert amq.device_status() == 0
@@ -416,6 +425,7 @@ def run_ours(args, wl):
             line["cpu_baseline"] = cpu_baseline(wl, unit)
             if not args.no_extras:
                 line["cpu_baseline_table6"] = cpu_baseline_table6()
+                line["cpu_baseline_batched"] = cpu_baseline_all_cores()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
@@ -423,7 +433,7 @@ def run_ours(args, wl):
         print(json.dumps(line))
 
 
-def _event_ms(torch, fn, flush, iters):
+def _event_ms(torch, fn, flush, iters, want_min=False):
     """Median device time of fn (one launch chain) with the L2 flushed, untimed, before every run."""
     times = []
     for i in range(iters):
@@ -434,6 +444,8 @@ def _event_ms(torch, fn, flush, iters):
         e.record()
         torch.cuda.synchronize()
         times.append(s.elapsed_time(e))
+    if want_min:
+        return float(np.median(times)), float(np.min(times))
     return float(np.median(times))
 
 
@@ -465,12 +477,12 @@ def cold_gemv(amq, torch, dev, flush, peak, peak_kind):
         y = torch.empty((1, m), device=dev)
         for _ in range(3):
             amq.binary_gemm(Wcodes, Walpha, xc, xb, n, y=y)
-        ms = _event_ms(torch, lambda: amq.binary_gemm(Wcodes, Walpha, xc, xb, n, y=y), flush, 10)
+        ms, ms_min = _event_ms(torch, lambda: amq.binary_gemm(Wcodes, Walpha, xc, xb, n, y=y), flush, 20, want_min=True)
         alg = Wcodes.numel() * 4 + Walpha.numel() * 4 + m * 4 + xc.numel() * 4
         gbs = alg / (ms * 1e-3) / 1e9
         out.append({"workload": "batch-1 binary GEMV %dx%d, k_w=%d, k_a=%d, packed planes %d MiB (random bits), cold" % (
                         m, n, k_w, k_a, Wcodes.numel() * 4 >> 20),
-                    "ms": ms, "bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": peak, "frac": gbs / peak,
+                    "ms": ms, "ms_min": ms_min, "bound": "hbm", "achieved": gbs, "unit": "GB/s", "peak": peak, "frac": gbs / peak,
                     "peak_kind": "of " + peak_kind, "frac_of_nominal_8000": gbs / 8000.0, "algorithmic_bytes": int(alg)})
         del Wcodes, Walpha, y
     return out
@@ -529,7 +541,9 @@ def batched_lines(amq, torch, dev, flush, hbm_peak, peak_kind):
     except Exception:
         bf16, tkind = 1590.0, "of fallback bf16 x 2"
     int8_tops = 2.0 * bf16
-    out = []
+    int8_measured = measured_int8_tops(torch, dev)
+    out = [{"workload": "dense int8 peak: torch._int_mm 8192 x 8192 x 8192 (library kernel), best of 10, CUDA events",
+            "bound": "tensor", "achieved": int8_measured, "unit": "TOP/s (int8)", "assumed_peak_2x_bf16": int8_tops}]
     for name in ("lstm1024_b64", "gru2048_b256", "proj32768_b512"):
         wl = synth.WORKLOADS[name]
         wpr = amq.words_per_row(wl.n)
@@ -546,7 +560,9 @@ def batched_lines(amq, torch, dev, flush, hbm_peak, peak_kind):
         out.append({"workload": "binary GEMM of %s: stacked M=%d, N=%d, K=%d bit positions" % (
                         name, wl.m * wl.k_w, wl.batch * wl.k_a, wpr * 32),
                     "ms": ms, "bound": "tensor", "achieved": tops, "unit": "TOP/s (int8, 2 per bit-MAC)", "peak": int8_tops,
-                    "frac": tops / int8_tops, "peak_kind": tkind, "bit_mac_per_s": mac / (ms * 1e-3)})
+                    "frac": tops / int8_tops, "peak_kind": tkind, "bit_mac_per_s": mac / (ms * 1e-3),
+                    "peak_int8_measured": int8_measured,
+                    "frac_of_int8_measured": (tops / int8_measured) if int8_measured else None})
         msq = _burst_ms(torch, lambda: amq.quantize(acts, wl.k_a, wl.T, codes=xc, coeffs=xb), 20)
         out.append({"workload": "on-line quantizer of %s: %d vectors of %d, k=%d, T=%d" % (name, wl.batch, wl.n, wl.k_a, wl.T),
                     "ms": msq, "bound": "latency"})
@@ -564,6 +580,28 @@ def batched_lines(amq, torch, dev, flush, hbm_peak, peak_kind):
     out.extend(table6_lines(amq, torch, dev, flush))
     out.append(quality_line(amq, torch, dev))
     return out
+
+
+def measured_int8_tops(torch, dev):
+    """Dense int8 throughput of this GPU as the library's own int8 matrix product reaches it (2 N^3 operations, best of
+    10): the denominator for the tensor-core lines next to the nominal 2 x bf16 figure.  None if the routine is missing."""
+    try:
+        n = 8192
+        a = torch.randint(-8, 8, (n, n), dtype=torch.int8, device=dev)
+        b = torch.randint(-8, 8, (n, n), dtype=torch.int8, device=dev)
+        for _ in range(3):
+            torch._int_mm(a, b)
+        best = 1e30
+        for _ in range(10):
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record()
+            torch._int_mm(a, b)
+            e.record()
+            torch.cuda.synchronize()
+            best = min(best, s.elapsed_time(e))
+        return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+    except Exception:
+        return None
 
 
 def paper_form_line(amq, torch, dev):
@@ -754,6 +792,60 @@ def cpu_baseline_table6():
         out.append({"workload": "Table 6 shape %d x 1024, %d/%d bits, batch 1: oracle on one host core" % (m, k, k),
                     "quantize_ms": 1e3 * best_q, "product_ms": 1e3 * best_p, "total_ms": 1e3 * (best_q + best_p),
                     "cores": 1, "kind": "oracle", "sample": "best of 3; weights quantized beforehand"})
+    return out
+
+
+def _oracle_worker(job):
+    """One process of the all-cores oracle runs: its share of the sequences (or of the weight rows)."""
+    name, lo, hi = job
+    import oracle
+    wl = synth.WORKLOADS[name]
+    ins = synth.inputs(wl)
+    if wl.cell == "proj":
+        W = synth.weights(wl, rows=hi)[lo:hi].astype(np.float64)
+        t0 = time.perf_counter()
+        Wc, Wa = oracle.quantize_rows(W, wl.k_w, wl.T)                      # the bulk quantization is part of this pass
+        Xc, Xb = oracle.quantize_rows(ins["acts"][:32].astype(np.float64), wl.k_a, wl.T)
+        oracle.binary_gemm(Wc, Wa, Xc, Xb, wl.n)
+        return time.perf_counter() - t0
+    Wc, Wa = oracle_setup(wl)
+    xs, h0, c0 = ins["x_seq"][:, lo:hi], ins["h0"][lo:hi], ins["c0"][lo:hi]
+    t0 = time.perf_counter()
+    if wl.cell == "lstm":
+        oracle.lstm_sequence(Wc, Wa, None, wl.I, wl.H, xs, h0, c0, wl.k_a, wl.T)
+    else:
+        oracle.gru_sequence(Wc, Wa, None, wl.I, wl.H, xs, h0, wl.k_a, wl.T)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline_all_cores():
+    """The oracle, as it stands, on ALL host cores for the batched workloads: independent sequences (weight rows for
+    the projection pass) are dealt out to one process per core; the time is that of the slowest process.  Bounded
+    samples: one sequence per core; for the projection 64 weight rows per core and 32 of the 512 activation vectors
+    (scaled to the whole pass by work)."""
+    import multiprocessing as mp
+    cores = os.cpu_count() or 1
+    out = []
+    ctx = mp.get_context("fork")
+    for name in ("lstm1024_b64", "gru2048_b256", "proj32768_b512"):
+        wl = synth.WORKLOADS[name]
+        per = 64 if wl.cell == "proj" else 1
+        jobs = [(name, c * per, (c + 1) * per) for c in range(cores)]
+        try:
+            with ctx.Pool(cores) as pool:
+                times = pool.map(_oracle_worker, jobs)
+        except Exception as exc:
+            out.append({"workload": name, "error": str(exc)[:120]})
+            continue
+        dt = max(times)
+        if wl.cell == "proj":
+            fraction = (cores * per / wl.m) * (32.0 / wl.batch)
+            out.append({"workload": name, "value": fraction / dt, "unit": "passes/s", "cores": cores, "kind": "oracle",
+                        "sample": "%d weight rows per core (quantized and multiplied), 32 of %d activation vectors; scaled by work"
+                                  % (per, wl.batch)})
+        else:
+            out.append({"workload": name, "value": cores * per * wl.steps / dt, "unit": "timesteps/s", "cores": cores,
+                        "kind": "oracle", "sample": "one full sequence (%d timesteps) per core; weight quantization not timed" % wl.steps})
     return out
 
 
