@@ -135,7 +135,10 @@ AMQ_API amq_status amq_binary_gemm(const uint32_t* Wcodes, const float* Walpha, 
  * Synchronises `stream`, then reads and clears the library's device-side status word of the current
  * device: AMQ_OK, or AMQ_ERR_TIMEOUT if a bounded wait inside a product kernel ran out since the last
  * read (the outputs of that call are then undefined).  Covers amq_binary_dots, amq_binary_gemm and the
- * product inside the cell calls; the sequence kernels report through amq_workspace_status as well.
+ * product inside the cell calls (amq_lstm_step_static included); the sequence kernels report through
+ * amq_workspace_status as well.  The word belongs to the device, not to a stream: a failure on any stream of the
+ * device is reported to whoever reads next (the read is one atomic swap enqueued on `stream`), and two host threads
+ * reading at the same time must be serialised by the caller.
  */
 AMQ_API amq_status amq_device_status(void* stream);
 
@@ -170,8 +173,9 @@ AMQ_API amq_status amq_lstm_step(const uint32_t* Wcodes, const float* Walpha, co
  *   - Arguments as for amq_lstm_step, without the workspace.  A problem whose scratch
  *     (amq_lstm_step_static_scratch_bytes) exceeds AMQ_STATIC_SCRATCH_BYTES is rejected with
  *     AMQ_ERR_WORKSPACE before anything is launched.
- *   - The first call on each device looks up the array's device address (once, with that device
- *     current); make that first call outside any stream capture.
+ *   - Every call looks up the array's device address for the device that is current at the call (`stream`
+ *     must belong to that device).  The first call on a device also makes the runtime load the library's
+ *     module there: make that first call outside any stream capture.
  *   - All calls on a device share the one array, which keeps whatever the last call left.  Each call
  *     rewrites the part it reads in full before reading it, so nothing needs clearing; but two calls
  *     whose work overlaps on the GPU (different streams, no ordering) race on it: order them.

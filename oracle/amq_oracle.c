@@ -99,7 +99,7 @@ int amq_oracle_ls_refit(const double* w, int n, int k, const int8_t* b, double* 
 }
 
 /* ---------------------------------------------------------------------------------------------
- * Level table (Algorithm 2, "construct v of all feasible codes in ascending order"):
+ * Level table (Algorithm 2, the step that lists every feasible code value in ascending order):
  * v_c = sum_i s_i(c) alpha_i for all 2^k codes, sorted ascending by (value, code index).
  * v and code have 2^k entries.
  * ------------------------------------------------------------------------------------------- */
@@ -121,27 +121,30 @@ void amq_oracle_levels(const double* alpha, int k, double* v, int* code)
 }
 
 /* ---------------------------------------------------------------------------------------------
- * Algorithm 1 (binary search tree): for one entry w and the ascending table v[lo..hi), halve the
- * range k times; go to the upper half when w >= (v[mid-1] + v[mid]) / 2.  Returns the position in v.
+ * Algorithm 1 (binary search tree over the ascending table v of 2^k levels), for one entry w: k
+ * levels of descent.  A node owns a window of table positions [first, first + 2 * half); the entry
+ * moves into the upper half of the window exactly when it is at least the midpoint between the
+ * largest level of the lower half and the smallest level of the upper half (so an entry on a
+ * midpoint goes up).  After k levels the window is one position: the level assigned to w.
  * ------------------------------------------------------------------------------------------- */
-static int bst_position(double w, const double* v, int lo, int hi)
+static int bst_position(double w, const double* v, int k)
 {
-    if (hi - lo == 1) return lo;
-    int mid = lo + (hi - lo) / 2;
-    double thr = (v[mid - 1] + v[mid]) / 2.0;
-    if (w >= thr) return bst_position(w, v, mid, hi);
-    return bst_position(w, v, lo, mid);
+    int first = 0;
+    for (int half = (1 << k) >> 1; half >= 1; half >>= 1) {
+        double boundary = 0.5 * (v[first + half - 1] + v[first + half]);
+        if (w >= boundary) first += half;
+    }
+    return first;
 }
 
 /* Code update of Algorithm 2 via Algorithm 1, for every entry, coefficients fixed. */
 void amq_oracle_bst(const double* w, int n, int k, const double* alpha, int8_t* b)
 {
-    int m = 1 << k;
     double v[1 << AMQ_ORACLE_MAX_K];
     int code[1 << AMQ_ORACLE_MAX_K];
     amq_oracle_levels(alpha, k, v, code);
     for (int t = 0; t < n; ++t) {
-        int c = code[bst_position(w[t], v, 0, m)];
+        int c = code[bst_position(w[t], v, k)];
         for (int i = 0; i < k; ++i) b[(size_t)i * n + t] = ((c >> (k - 1 - i)) & 1) ? 1 : -1;
     }
 }
@@ -392,7 +395,7 @@ void amq_oracle_lstm_step(const uint32_t* Wcodes, const double* Walpha, const do
 /* ---------------------------------------------------------------------------------------------
  * One quantized LSTM step in the form the paper states it (Eq. 6 and the text after it): two weight
  * matrices W_i (4H x I) and W_h (4H x H), each quantized row by row on its own; x_t is a row of the
- * quantized embedding W_e and "needs no more quantization", so it arrives as k_e packed planes with
+ * quantized embedding W_e and is used as it is (Sec. 4), so it arrives as k_e packed planes with
  * coefficients; only h_{t-1} is quantized on-line (k_a bits, T cycles).
  *   p = W_i_hat x_hat + W_h_hat h_hat + bias;  i, f, o = logistic(p), g = tanh(p) (gate order i, f, o, g);
  *   c' = f * c + i * g;  h' = o * tanh(c').

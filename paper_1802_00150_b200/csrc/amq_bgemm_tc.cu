@@ -48,6 +48,7 @@ constexpr int MAX_STAGES = 4;
 constexpr unsigned WAIT_LIMIT = 1u << 20;   // attempts on an mbarrier before giving up
 
 __device__ uint32_t g_tc_status;            // nonzero after a bounded wait ran out (sticky until read)
+__device__ uint32_t g_tc_status_taken;      // what the last read found
 
 struct TcParams {
     GemmArgs a;
@@ -808,17 +809,14 @@ struct TcPlan {
     bool persistent;
 };
 
+// SMs of the current device (asked every time: an attribute query costs well under a microsecond and the answer
+// belongs to the device that is current now, not to the one that was current at the first call)
 int sm_count()
 {
-    static int count = 0;       // the same on every device of a node
-    if (count == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-            count = v;
-        else
-            return 148;
-    }
-    return count;
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+        return v;
+    return 1;
 }
 
 // The persistent form: one M tile per CTA step, dedicated epilogue warps, two accumulator buffers when they fit tensor
@@ -886,7 +884,7 @@ bool plan(const GemmArgs& a, TcPlan* out)
     for (int sft = 0; sft < 8; ++sft) p.mul[sft] = 1u << (7 - sft);
     p.mask_sign = 0x80808080u;
     p.mask_half = 0x40404040u;
-    p.MT = (2 * p.nseg * p.n_mma <= 512 && (long long)(mtiles / 2) * btiles >= 2 * 148) ? 2 : 1;
+    p.MT = (2 * p.nseg * p.n_mma <= 512 && (long long)(mtiles / 2) * btiles >= 2 * sm_count()) ? 2 : 1;
     // with one M tile per CTA and more tiles than SMs, the persistent form hides the epilogues; with two M tiles
     // per CTA the plain form's lower shared-memory traffic per MMA counts for more (measured)
     if (p.MT == 1 && plan_persistent(p, mtiles, btiles, out)) return true;
@@ -963,14 +961,19 @@ amq_status launch_binary_gemm_tc(const GemmArgs& a, cudaStream_t st)
     return AMQ_ERR_UNSUPPORTED;
 }
 
+// one thread swaps the status word for zero and leaves the old value in the second word: read and clear are a single
+// atomic step, so a failure recorded by a kernel of another stream in between is neither lost nor reported twice
+__global__ void take_tc_status_kernel()
+{
+    g_tc_status_taken = atomicExch(&g_tc_status, 0u);
+}
+
 amq_status read_tc_status(cudaStream_t st, uint32_t* out)
 {
+    take_tc_status_kernel<<<1, 1, 0, st>>>();
+    AMQ_LAUNCH_CHECK();
     AMQ_CUDA_TRY(cudaStreamSynchronize(st));
-    AMQ_CUDA_TRY(cudaMemcpyFromSymbol(out, g_tc_status, sizeof(uint32_t)));
-    if (*out) {
-        const uint32_t zero = 0;
-        AMQ_CUDA_TRY(cudaMemcpyToSymbol(g_tc_status, &zero, sizeof(uint32_t)));
-    }
+    AMQ_CUDA_TRY(cudaMemcpyFromSymbol(out, g_tc_status_taken, sizeof(uint32_t)));
     return AMQ_OK;
 }
 

@@ -1,6 +1,6 @@
 // Quantized LSTM in the form the paper states it (Eq. 6 and the paragraph after it): two weight matrices
 // W_i (4H x I) and W_h (4H x H), each quantized row by row on its own; the input x_t is a row of the quantized
-// embedding matrix and "needs no more quantization" (it arrives as packed planes + coefficients, see
+// embedding matrix and is used as it is, without a second quantization (it arrives as packed planes + coefficients, see
 // amq_embedding_rows); only h_{t-1} is quantized on-line.
 //
 // Because x_t does not depend on the recurrent state, the input projections W_i x_t + b of ALL timesteps of

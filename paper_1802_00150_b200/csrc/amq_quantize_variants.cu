@@ -4,6 +4,7 @@
 // for generality, not speed: one warp per row, elements 32 q + lane, every pass re-reads the row (it stays in
 // L1/L2), the sign planes live in shared memory in the packed layout (a warp ballot IS word q of a plane).
 #include "amq_common.cuh"
+#include "amq_quantize_device.cuh"
 
 namespace amq {
 namespace {
@@ -18,12 +19,31 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-// Eq. 5 on the first kk planes: G = B^T B from popcounts (exact), c = B^T w, solved in fp64 by Gaussian
-// elimination with partial pivoting; a pivot below 1e-9 n leaves alpha untouched.  Every lane runs the same solve.
+// solve_refit of the production quantizer on the first KK coefficients of alpha[]
+template <int KK>
+__device__ __forceinline__ void solve_first(const float* c, const int* gram, int n, float* alpha)
+{
+    float cc[KK], aa[KK];
+    int gg[KK > 1 ? KK * (KK - 1) / 2 : 1];
+#pragma unroll
+    for (int i = 0; i < KK; ++i) { cc[i] = c[i]; aa[i] = alpha[i]; }
+#pragma unroll
+    for (int q = 0; q < (KK > 1 ? KK * (KK - 1) / 2 : 1); ++q) gg[q] = gram[q];
+    if (solve_refit<KK>(cc, gg, n, aa)) {
+#pragma unroll
+        for (int i = 0; i < KK; ++i) alpha[i] = aa[i];
+    }
+}
+
+// Eq. 5 on the first kk planes: G = B^T B from popcounts (exact integers, upper triangle in row-major order),
+// c = B^T w, then the solve of the production quantizer (a singular system leaves alpha untouched).  Every lane
+// runs the same solve.
 __device__ void refit(const float* __restrict__ x, int n, int kk, const uint32_t (*planes)[VAR_MAX_WORDS], int lane, float* alpha)
 {
     const int Q = (n + 31) >> 5;
-    double G[AMQ_MAX_K][AMQ_MAX_K + 1];
+    float c[AMQ_MAX_K];
+    int gram[AMQ_MAX_K * (AMQ_MAX_K - 1) / 2];
+    int g = 0;
     for (int i = 0; i < kk; ++i) {
         for (int j = i + 1; j < kk; ++j) {
             int diff = 0;
@@ -31,38 +51,22 @@ __device__ void refit(const float* __restrict__ x, int n, int kk, const uint32_t
                 const uint32_t mask = (32 * q + 32 <= n) ? 0xffffffffu : ((1u << (n - 32 * q)) - 1u);
                 diff += __popc((planes[i][q] ^ planes[j][q]) & mask);
             }
-            diff = __reduce_add_sync(0xffffffffu, diff);
-            G[i][j] = G[j][i] = (double)(n - 2 * diff);
+            gram[g++] = n - 2 * __reduce_add_sync(0xffffffffu, diff);
         }
-        G[i][i] = (double)n;
-        float c = 0.0f;
+        float ci = 0.0f;
         for (int q = 0; q < Q; ++q) {
             const int t = 32 * q + lane;
             const float w = t < n ? x[t] : 0.0f;
-            c += ((planes[i][q] >> lane) & 1u) ? w : -w;
+            ci += ((planes[i][q] >> lane) & 1u) ? w : -w;
         }
-        G[i][kk] = (double)warp_sum(c);
+        c[i] = warp_sum(ci);
     }
-    const double tiny = 1e-9 * (double)n;
-    for (int col = 0; col < kk; ++col) {
-        int piv = col;
-        for (int row = col + 1; row < kk; ++row)
-            if (fabs(G[row][col]) > fabs(G[piv][col])) piv = row;
-        if (!(fabs(G[piv][col]) >= tiny) || fabs(G[piv][col]) == 0.0) return;
-        if (piv != col)
-            for (int j = 0; j <= kk; ++j) { const double tmp = G[col][j]; G[col][j] = G[piv][j]; G[piv][j] = tmp; }
-        for (int row = col + 1; row < kk; ++row) {
-            const double f = G[row][col] / G[col][col];
-            for (int j = col; j <= kk; ++j) G[row][j] -= f * G[col][j];
-        }
+    switch (kk) {
+        case 1: solve_first<1>(c, gram, n, alpha); break;
+        case 2: solve_first<2>(c, gram, n, alpha); break;
+        case 3: solve_first<3>(c, gram, n, alpha); break;
+        case 4: solve_first<4>(c, gram, n, alpha); break;
     }
-    double sol[AMQ_MAX_K];
-    for (int i = kk - 1; i >= 0; --i) {
-        double s = G[i][kk];
-        for (int j = i + 1; j < kk; ++j) s -= G[i][j] * sol[j];
-        sol[i] = s / G[i][i];
-    }
-    for (int i = 0; i < kk; ++i) alpha[i] = (float)sol[i];
 }
 
 __global__ void __launch_bounds__(VAR_WARPS * 32)

@@ -9,10 +9,10 @@
 //
 // The array lives in the data segment of every device that loads the library (AMQ_STATIC_SCRATCH_BYTES per
 // GPU, until the process exits).  In host code the array's name is only a host-side handle, not a device
-// address, so the address is looked up once per device with cudaGetSymbolAddress and handed to the
-// kernels as an ordinary pointer.
-#include <mutex>
-
+// address, so the address is looked up with cudaGetSymbolAddress (for the device that is current at the
+// call) and handed to the kernels as an ordinary pointer.  The lookup is repeated on every call: once the
+// module is loaded it is a table lookup, and an address remembered from an earlier call would be stale after
+// the application reset the device or tore its context down.
 #include "amq_common.cuh"
 
 namespace amq {
@@ -21,24 +21,13 @@ namespace {
 
 static __device__ __align__(256) unsigned char g_static_scratch[AMQ_STATIC_SCRATCH_BYTES];
 
-constexpr int MAX_DEVICES = 64;
-std::mutex g_scratch_mutex;
-unsigned char* g_scratch_ptr[MAX_DEVICES];      // device address of g_static_scratch, per device ordinal
-
-// Device address of the scratch array on the current device; looked up on the first call per device.
+// Device address of the scratch array on the current device.
 amq_status static_scratch(unsigned char** out)
 {
-    int dev = 0;
-    AMQ_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= MAX_DEVICES) return AMQ_ERR_UNSUPPORTED;
-    std::lock_guard<std::mutex> lock(g_scratch_mutex);
-    if (!g_scratch_ptr[dev]) {
-        void* p = nullptr;
-        AMQ_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
-        if (!p) return AMQ_ERR_CUDA;
-        g_scratch_ptr[dev] = static_cast<unsigned char*>(p);
-    }
-    *out = g_scratch_ptr[dev];
+    void* p = nullptr;
+    AMQ_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+    if (!p) return AMQ_ERR_CUDA;
+    *out = static_cast<unsigned char*>(p);
     return AMQ_OK;
 }
 
