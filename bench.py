@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by workload; the summaries are under profiles/.  None = not captured for the
 # kernel as it stands.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"lstm1024_b1": 2422016 + 51968}    # rnn_persistent_kernel, profiles/rnn_persistent_kernel_lstm1024_b1.txt
 # the same for the cold matrix-vector kernel on 131072 x 8192 at 2/2 bits (profiles/bgemv_kernel_131072x8192_k2k2.txt)
 NCU_TRAFFIC_GEMV_COLD_BYTES = 269500000
 
@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the cold-GEMV bandwidth lines and the batched-regime lines")
+    ap.add_argument("--phase-timing", action="store_true",
+                    help="build the library with per-phase clock counters in the batch-1 sequence kernel, run the workload "
+                         "with it and print the per-phase table instead of the benchmark line (not a benchmark value)")
     return ap.parse_args()
 
 
@@ -866,9 +869,44 @@ def cpu_baseline(wl, unit):
             "sample": "%d x %s; fp64, single thread; weight quantization not timed" % (reps, desc)}
 
 
+def run_phase_timing(args, wl):
+    """Per-phase SM clocks per timestep of the batch-1 sequence kernel (first and last CTA), from a build of the library
+    with AMQ_PHASE_TIMING defined: phases = gather (x loads + waiting for the other CTAs' h), on-line quantizer,
+    packing + barrier, product + gates + publish (thread 0, whose warp owns the CTA's first hidden unit)."""
+    from paper_1802_00150_b200 import build
+    lib = build.build(defines=["AMQ_PHASE_TIMING"], lib_name="libamq_b200_phase.so")
+    os.environ["AMQ_B200_LIBRARY"] = lib
+    import torch
+    from paper_1802_00150_b200 import amq
+    assert wl.batch == 1 and wl.cell in ("lstm", "gru"), "the phase counters are in the batch-1 sequence kernel"
+    if wl.steps == 1:
+        wl = synth.scaled(wl, steps=35)
+    dev = torch.device("cuda", 0)
+    Wcodes, Walpha = amq.quantize(torch.from_numpy(synth.weights(wl)).to(dev), wl.k_w, wl.T)
+    ins = synth.inputs(wl)
+    x_seq = torch.from_numpy(ins["x_seq"]).to(dev)
+    h0, c0 = torch.from_numpy(ins["h0"]).to(dev), torch.from_numpy(ins["c0"]).to(dev)
+    ws = amq.new_workspace(wl.I, wl.H, 1, wl.k_a)
+    for _ in range(max(args.warmup, 3)):
+        if wl.cell == "lstm":
+            amq.lstm_sequence(Wcodes, Walpha, None, wl.I, wl.H, x_seq, h0, c0, wl.k_a, wl.T, ws)
+        else:
+            amq.gru_sequence(Wcodes, Walpha, None, wl.I, wl.H, x_seq, h0, wl.k_a, wl.T, ws)
+    torch.cuda.synchronize()
+    words = ws.cpu().numpy().view(np.uint32)
+    names = ["gather", "quantize", "pack", "product_gates_publish"]
+    print(json.dumps({"workload": wl.name, "timesteps": wl.steps, "unit": "SM clocks per timestep, thread 0",
+                      "first_cta": dict(zip(names, (int(v) for v in words[8:12]))),
+                      "last_cta": dict(zip(names, (int(v) for v in words[16:20]))),
+                      "sum_first_cta": int(words[8:12].sum())}))
+
+
 def main():
     args = parse_args()
     wl = synth.WORKLOADS[args.workload]
+    if args.phase_timing:
+        run_phase_timing(args, wl)
+        return
     if args.impl == "reference":
         run_reference(args, wl)
     else:

@@ -10,7 +10,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libamq_b200.so")
+# the product library; AMQ_B200_LIBRARY names an instrumented build of the same sources instead (see build.py)
+LIB_PATH = os.environ.get("AMQ_B200_LIBRARY") or os.path.join(_HERE, "libamq_b200.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
