@@ -132,6 +132,22 @@ AMQ_API amq_status amq_binary_gemm(const uint32_t* Wcodes, const float* Walpha, 
                            const float* bias, float* y, int ldy, void* stream);
 
 /*
+ * The operation Table 6 (Appendix A) times, in one launch: on-line quantization of ONE activation vector (Sec. 4: the
+ * hidden state is quantized during inference) followed by the binary matrix-vector product with row-wise quantized
+ * weights,
+ *   (beta, x_j) = Algorithm 2 on x with k_a bits and T cycles;  y[r] = sum_i sum_j Walpha[r][i] beta[j] D[r][i][j] + bias[r].
+ * x [n] DEVICE fp32, n <= 2048 (longer vectors: amq_quantize, then amq_binary_gemm; AMQ_ERR_UNSUPPORTED here);
+ * Wcodes [m][k_w][wpr], Walpha [m][k_w], bias [m] or NULL, y [m] fp32 out.  xcodes_out [k_a][wpr] (16-byte aligned) and
+ * xbeta_out [k_a], each may be NULL: the planes and coefficients of the quantized vector, for a caller that needs them
+ * again (a recurrent product on the same state).  Every CTA of the product quantizes the vector for itself; the
+ * arithmetic and the readings of amq_quantize apply (a different but equally fixed summation order, so codes of
+ * elements on a decision boundary may differ from amq_quantize's; results repeat bit for bit from run to run).
+ */
+AMQ_API amq_status amq_quantized_gemv(const uint32_t* Wcodes, const float* Walpha, int m, int n, int k_w,
+                              const float* x, int k_a, int T, const float* bias, float* y,
+                              uint32_t* xcodes_out, float* xbeta_out, void* stream);
+
+/*
  * Synchronises `stream`, then reads and clears the library's device-side status word of the current
  * device: AMQ_OK, or AMQ_ERR_TIMEOUT if a bounded wait inside a product kernel ran out since the last
  * read (the outputs of that call are then undefined).  Covers amq_binary_dots, amq_binary_gemm and the

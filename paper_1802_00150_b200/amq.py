@@ -37,6 +37,7 @@ EXPORTS = {
     "amq_unpack": (_int, [_vp, _vp, _int, _int, _int, _vp, _vp]),
     "amq_binary_dots": (_int, [_vp, _int, _int, _int, _vp, _int, _int, _vp, _vp]),
     "amq_binary_gemm": (_int, [_vp, _vp, _int, _int, _int, _vp, _vp, _int, _int, _vp, _vp, _int, _vp]),
+    "amq_quantized_gemv": (_int, [_vp, _vp, _int, _int, _int, _vp, _int, _int, _vp, _vp, _vp, _vp, _vp]),
     "amq_device_status": (_int, [_vp]),
     "amq_cell_workspace_bytes": (_sz, [_int, _int, _int, _int]),
     "amq_cell_host_staging_bytes": (_sz, [_int, _int, _int, _int]),
@@ -177,6 +178,22 @@ def binary_gemm(Wcodes, Walpha, xcodes, xbeta, n, bias=None, y=None):
     _check(_lib.amq_binary_gemm(_ptr(Wcodes), _ptr(Walpha), m, n, k_w, _ptr(xcodes), _ptr(xbeta), batch, k_a,
                                 _ptr(bias), _ptr(y), y.stride(0) if batch > 1 else max(m, y.stride(0)), _stream()))
     return y
+
+
+def quantized_gemv(Wcodes, Walpha, x, k_a, T, bias=None, y=None, want_codes=False):
+    """Table 6's operation in one launch: x (n,) or (1, n) fp32 is quantized on-line (k_a bits, T cycles) inside the
+    product kernel.  Returns y (m,), or (y, xcodes (k_a, wpr), xbeta (k_a,)) with want_codes."""
+    Wcodes, Walpha = _dev(Wcodes, torch.int32, "Wcodes"), _dev(Walpha, torch.float32, "Walpha")
+    x = _dev(x, torch.float32, "x")
+    m, k_w, wpr = Wcodes.shape
+    n = x.numel()
+    if y is None:
+        y = torch.empty((m,), dtype=torch.float32, device=x.device)
+    xc = torch.empty((k_a, wpr), dtype=torch.int32, device=x.device) if want_codes else None
+    xb = torch.empty((k_a,), dtype=torch.float32, device=x.device) if want_codes else None
+    _check(_lib.amq_quantized_gemv(_ptr(Wcodes), _ptr(Walpha), m, n, k_w, _ptr(x), k_a, T, _ptr(bias), _ptr(y),
+                                   _ptr(xc), _ptr(xb), _stream()))
+    return (y, xc, xb) if want_codes else y
 
 
 def device_status():

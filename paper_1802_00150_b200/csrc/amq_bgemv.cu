@@ -11,7 +11,14 @@
 // Bit counting is the second ceiling right behind the memory one (one POPC per weight word and
 // activation plane issues at a quarter of the logic rate), so pairs of XOR-ed words first go through a
 // carry-save adder on whole words (two LOP3) and only the carries and the final sums are counted.
+//
+// Fused form (the operation Table 6 times: on-line quantization of the activation vector, then the product, in ONE
+// launch): every CTA quantizes the fp32 vector itself (Algorithm 2 with the CTA as the group, the same device code as
+// the recurrent kernel; redundant across CTAs, which costs a microsecond of latency and no memory traffic worth
+// naming) into shared memory and takes its activation planes from there; its first weight rows are already in flight
+// meanwhile.  For vectors of up to 2048 elements.
 #include "amq_common.cuh"
+#include "amq_quantize_device.cuh"
 
 namespace amq {
 
@@ -28,7 +35,15 @@ struct GemvParams {
     int m, n, CH;
     int epilogue;
     bool overlap;               // host side only: launch as a programmatic dependent of the preceding kernel
+    // fused form: the fp32 vector, alternating cycles, and where CTA 0 leaves the planes and coefficients (or null)
+    const float* xf;
+    int T;
+    uint32_t* xcodes_out;
+    float* xbeta_out;
 };
+
+constexpr int FQ_EPT = 8;       // fused form: 256 threads x 8 consecutive elements each
+constexpr int FQ_MAX_CH = 16;   // = 2048 bit positions
 
 // differing bits of (w xor x) over the four words of a chunk, accumulated carry-save:
 // `ones` carries the bit-wise sums, the return value counts the carries (weight 2)
@@ -61,11 +76,13 @@ __device__ __forceinline__ int segment_sum(int v)
 // never drains while a warp computes.  After the segment sums every lane of a segment holds the totals of
 // that segment's row; lane `sub` of segment `seg` keeps the ones of row sub * (32 / SEG) + seg, and when
 // the block is complete all 32 lanes fold coefficients and bias and store 32 consecutive outputs at once.
-template <int KW, int KA, int CPT, int R, int SEG_LOG2, bool EXACT>
+template <int KW, int KA, int CPT, int R, int SEG_LOG2, bool EXACT, bool FQ>
 __global__ void __launch_bounds__(256)
 bgemv_kernel(GemvParams p)
 {
-    grid_dependency_wait();     // the activation planes may come from the preceding kernel of the stream
+    __shared__ __align__(16) uint4 sX[FQ ? KA : 1][FQ ? FQ_MAX_CH : 1];
+    __shared__ QuantScratch<KA, FQ ? 8 : 1> q_scratch;
+    if (!FQ) grid_dependency_wait();     // the activation planes may come from the preceding kernel of the stream
     const int lane = threadIdx.x & 31;
     constexpr int SEG = 1 << SEG_LOG2;
     constexpr int spw = 32 >> SEG_LOG2;            // rows per load instruction of the warp
@@ -75,19 +92,11 @@ bgemv_kernel(GemvParams p)
     const int CH = EXACT ? CPT * SEG : p.CH;
     const size_t row_chunks = (size_t)KW * CH;
 
-    // activation planes of this lane's columns
-    uint4 xr[KA][CPT];
     bool has[CPT];
 #pragma unroll
-    for (int c = 0; c < CPT; ++c) {
-        has[c] = EXACT || (sub + c * SEG < CH);
-#pragma unroll
-        for (int j = 0; j < KA; ++j)
-            xr[j][c] = has[c] ? p.x[(size_t)j * CH + sub + c * SEG] : make_uint4(0, 0, 0, 0);   // ordinary load, L1-cached
-    }
+    for (int c = 0; c < CPT; ++c) has[c] = EXACT || (sub + c * SEG < CH);
+    uint4 xr[KA][CPT];          // activation planes of this lane's columns, and their coefficients (filled below)
     float beta[KA];
-#pragma unroll
-    for (int j = 0; j < KA; ++j) beta[j] = (p.epilogue == EPI_Y) ? p.xbeta[j] : 0.0f;
 
     const long long blocks = ((long long)p.m + 31) >> 5;
     const long long warp_global = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -175,7 +184,55 @@ bgemv_kernel(GemvParams p)
     };
 
     uint4 wa[R][KW][CPT], wb[R][KW][CPT];
-    if (g < g_end) load_pass(wa, g / PASSES, (int)(g % PASSES));
+    if (g < g_end) load_pass(wa, g / PASSES, (int)(g % PASSES));     // weights are constant: in flight before anything else
+
+    if constexpr (FQ) {
+        // on-line quantization of the vector by this CTA: thread t owns the 8 consecutive elements 8 t .. 8 t + 7, so
+        // the sign bits the quantizer leaves in a register are byte t of the packed plane
+        quant_scratch_init(q_scratch);
+        grid_dependency_wait();                            // the vector may come from the preceding kernel of the stream
+        const int tid = threadIdx.x, e0 = tid * FQ_EPT;
+        float w[FQ_EPT];
+        uint32_t valid = 0;
+#pragma unroll
+        for (int j = 0; j < FQ_EPT; ++j) {
+            const bool ok = e0 + j < p.n;
+            w[j] = ok ? __ldcg(p.xf + e0 + j) : 0.0f;
+            valid |= (ok ? 1u : 0u) << j;
+        }
+        uint32_t bits[KA];
+        quantize_group<KA, FQ_EPT, 8>(w, valid, p.n, quant_padding_consecutive(p.n, FQ_EPT), p.T, beta, bits, q_scratch);
+        if (e0 < CH * 128) {
+#pragma unroll
+            for (int j = 0; j < KA; ++j) reinterpret_cast<uint8_t*>(&sX[j][0])[tid] = (uint8_t)bits[j];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int c = 0; c < CPT; ++c)
+#pragma unroll
+            for (int j = 0; j < KA; ++j) xr[j][c] = has[c] ? sX[j][sub + c * SEG] : make_uint4(0, 0, 0, 0);
+        if (blockIdx.x == 0 && p.xcodes_out) {             // the planes and coefficients, for whoever needs them next
+            for (int q = tid; q < KA * CH * 4; q += blockDim.x) {
+                const int j = q / (CH * 4), wq = q - j * CH * 4;
+                p.xcodes_out[q] = reinterpret_cast<const uint32_t*>(&sX[j][0])[wq];
+            }
+            if (tid < KA && p.xbeta_out) {
+                float b = beta[0];
+#pragma unroll
+                for (int j = 1; j < KA; ++j) b = (tid == j) ? beta[j] : b;
+                p.xbeta_out[tid] = b;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int c = 0; c < CPT; ++c)
+#pragma unroll
+            for (int j = 0; j < KA; ++j)
+                xr[j][c] = has[c] ? p.x[(size_t)j * CH + sub + c * SEG] : make_uint4(0, 0, 0, 0);   // ordinary load, L1-cached
+#pragma unroll
+        for (int j = 0; j < KA; ++j) beta[j] = (p.epilogue == EPI_Y) ? p.xbeta[j] : 0.0f;
+    }
+
     while (g < g_end) {
         step(wa, wb);
         if (!(g < g_end)) break;
@@ -183,14 +240,14 @@ bgemv_kernel(GemvParams p)
     }
 }
 
-template <int KW, int KA, int CPT, int SEG_LOG2>
+template <int KW, int KA, int CPT, int SEG_LOG2, bool FQ>
 amq_status launch_cfg(const GemvParams& p, cudaStream_t st)
 {
     constexpr int SEG = 1 << SEG_LOG2;
     constexpr int R0 = (8 / (KW * CPT)) > 0 ? (8 / (KW * CPT)) : 1;     // about eight 128-bit loads per lane and pass
     constexpr int R = R0 < SEG ? R0 : SEG;
     const bool exact = p.CH == CPT * SEG;
-    auto kernel = exact ? bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, true> : bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, false>;
+    auto kernel = exact ? bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, true, FQ> : bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, false, FQ>;
     static thread_local int cached_dev = -1, cached_grid[2] = {0, 0};
     int dev = 0;
     AMQ_CUDA_TRY(cudaGetDevice(&dev));
@@ -199,8 +256,8 @@ amq_status launch_cfg(const GemvParams& p, cudaStream_t st)
         AMQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
         for (int e = 0; e < 2; ++e) {
             int per_sm = 0;
-            if (e) AMQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, true>, 256, 0));
-            else AMQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, false>, 256, 0));
+            if (e) AMQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, true, FQ>, 256, 0));
+            else AMQ_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, false, FQ>, 256, 0));
             cached_grid[e] = sms * (per_sm > 0 ? per_sm : 1);
         }
         cached_dev = dev;
@@ -219,11 +276,17 @@ amq_status launch_cfg(const GemvParams& p, cudaStream_t st)
 template <int KW, int KA>
 amq_status launch_cpt(const GemvParams& p, cudaStream_t st)
 {
-    if (p.CH <= 2) return launch_cfg<KW, KA, 1, 1>(p, st);
-    if (p.CH <= 8) return launch_cfg<KW, KA, 1, 3>(p, st);
-    if (p.CH <= 16) return launch_cfg<KW, KA, 1, 4>(p, st);
-    if (p.CH <= 32) return launch_cfg<KW, KA, 1, 5>(p, st);
-    return launch_cfg<KW, KA, 2, 5>(p, st);
+    if (p.xf) {                 // fused form: up to 16 chunks
+        if (p.CH <= 2) return launch_cfg<KW, KA, 1, 1, true>(p, st);
+        if (p.CH <= 8) return launch_cfg<KW, KA, 1, 3, true>(p, st);
+        if (p.CH <= FQ_MAX_CH) return launch_cfg<KW, KA, 1, 4, true>(p, st);
+        return AMQ_ERR_UNSUPPORTED;
+    }
+    if (p.CH <= 2) return launch_cfg<KW, KA, 1, 1, false>(p, st);
+    if (p.CH <= 8) return launch_cfg<KW, KA, 1, 3, false>(p, st);
+    if (p.CH <= 16) return launch_cfg<KW, KA, 1, 4, false>(p, st);
+    if (p.CH <= 32) return launch_cfg<KW, KA, 1, 5, false>(p, st);
+    return launch_cfg<KW, KA, 2, 5, false>(p, st);
 }
 
 template <int KW>
@@ -234,6 +297,17 @@ amq_status launch_ka(const GemvParams& p, int k_a, cudaStream_t st)
         case 2: return launch_cpt<KW, 2>(p, st);
         case 3: return launch_cpt<KW, 3>(p, st);
         case 4: return launch_cpt<KW, 4>(p, st);
+    }
+    return AMQ_ERR_UNSUPPORTED;
+}
+
+amq_status launch_kw(const GemvParams& p, int k_w, int k_a, cudaStream_t st)
+{
+    switch (k_w) {
+        case 1: return launch_ka<1>(p, k_a, st);
+        case 2: return launch_ka<2>(p, k_a, st);
+        case 3: return launch_ka<3>(p, k_a, st);
+        case 4: return launch_ka<4>(p, k_a, st);
     }
     return AMQ_ERR_UNSUPPORTED;
 }
@@ -259,13 +333,41 @@ amq_status launch_binary_gemv(const GemmArgs& a, cudaStream_t st)
     p.m = a.m; p.n = a.n; p.CH = words_per_row(a.n) / 4;
     p.epilogue = a.epilogue;
     p.overlap = a.overlap_with_previous;
-    switch (a.k_w) {
-        case 1: return launch_ka<1>(p, a.k_a, st);
-        case 2: return launch_ka<2>(p, a.k_a, st);
-        case 3: return launch_ka<3>(p, a.k_a, st);
-        case 4: return launch_ka<4>(p, a.k_a, st);
-    }
-    return AMQ_ERR_UNSUPPORTED;
+    p.xf = nullptr; p.T = 0; p.xcodes_out = nullptr; p.xbeta_out = nullptr;
+    return launch_kw(p, a.k_w, a.k_a, st);
+}
+
+bool quantized_gemv_supported(int n) { return n >= 1 && words_per_row(n) / 4 <= FQ_MAX_CH; }
+
+amq_status launch_quantized_gemv(const uint32_t* Wcodes, const float* Walpha, int m, int n, int k_w, const float* x, int k_a, int T,
+                                 const float* bias, float* y, uint32_t* xcodes_out, float* xbeta_out, cudaStream_t st,
+                                 bool overlap_with_previous)
+{
+    if (!quantized_gemv_supported(n)) return AMQ_ERR_UNSUPPORTED;
+    GemvParams p;
+    p.W = reinterpret_cast<const uint4*>(Wcodes);
+    p.Walpha = Walpha;
+    p.x = nullptr; p.xbeta = nullptr;
+    p.bias = bias;
+    p.y = y; p.D = nullptr;
+    p.m = m; p.n = n; p.CH = words_per_row(n) / 4;
+    p.epilogue = EPI_Y;
+    p.overlap = overlap_with_previous;
+    p.xf = x; p.T = T; p.xcodes_out = xcodes_out; p.xbeta_out = xbeta_out;
+    return launch_kw(p, k_w, k_a, st);
 }
 
 }  // namespace amq
+
+extern "C" amq_status amq_quantized_gemv(const uint32_t* Wcodes, const float* Walpha, int m, int n, int k_w,
+                                         const float* x, int k_a, int T, const float* bias, float* y,
+                                         uint32_t* xcodes_out, float* xbeta_out, void* stream)
+{
+    if (m < 0 || n < 1) return AMQ_ERR_INVALID_ARG;
+    if (!amq::valid_k(k_w) || !amq::valid_k(k_a) || T < 0 || !amq::quantized_gemv_supported(n)) return AMQ_ERR_UNSUPPORTED;
+    if (m == 0) return AMQ_OK;
+    if (!Wcodes || !Walpha || !x || !y) return AMQ_ERR_INVALID_ARG;
+    if (!amq::aligned16(Wcodes) || (xcodes_out && !amq::aligned16(xcodes_out))) return AMQ_ERR_ALIGNMENT;
+    return amq::launch_quantized_gemv(Wcodes, Walpha, m, n, k_w, x, k_a, T, bias, y, xcodes_out, xbeta_out,
+                                      (cudaStream_t)stream, false);
+}

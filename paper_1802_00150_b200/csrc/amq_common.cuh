@@ -141,6 +141,12 @@ amq_status launch_log_softmax_argmax(const float* logits, int rows, int n, int l
                                      cudaStream_t st, bool overlap_with_previous);
 bool gemv_supported(const GemmArgs& a);
 amq_status launch_binary_gemv(const GemmArgs& a, cudaStream_t st);
+// Fused form for one vector of up to 2048 elements: on-line quantization (k_a bits, T cycles) inside the product kernel;
+// xcodes_out [k_a][wpr] / xbeta_out [k_a] (may be null) receive the planes and coefficients.
+bool quantized_gemv_supported(int n);
+amq_status launch_quantized_gemv(const uint32_t* Wcodes, const float* Walpha, int m, int n, int k_w, const float* x, int k_a, int T,
+                                 const float* bias, float* y, uint32_t* xcodes_out, float* xbeta_out, cudaStream_t st,
+                                 bool overlap_with_previous);
 
 // Tensor-core kernel (tcgen05, batch >= 16): whether it covers a problem, its launch, and its status word
 // (nonzero after a bounded device-side wait ran out; cleared by the read).

@@ -2,7 +2,8 @@
 // as one chain on the caller's stream: per token the embedding row (pre-quantized, needs no further quantization),
 // the input projection W_i x + b, the recurrent product W_h h_hat on the on-line quantized state, the gates, the
 // quantizer on the new state (its planes serve the output layer now and the recurrence of the next token), the
-// output product W_s h_hat + b_s and log-softmax / arg-max.  Seven launches per token, no host round trip.
+// output product W_s h_hat + b_s and log-softmax / arg-max.  Six launches per token (the quantizer on the new state
+// runs inside the output product's kernel when the state has at most 2048 elements, else seven), no host round trip.
 #include "amq_common.cuh"
 
 namespace amq {
@@ -88,9 +89,16 @@ amq_status amq_lm_greedy_decode(const uint32_t* We_codes, const float* We_alpha,
         if (s != AMQ_OK) break;
         s = amq::launch_lstm_gates(ws.pre, ws.proj, c, h, c, H, st, true);                  // state updated in place
         if (s != AMQ_OK) break;
-        s = amq::launch_quantize(h, H, H, nullptr, 0, 0, 1, k_a, T, ws.hcodes, ws.hbeta, st, true);
-        if (s != AMQ_OK) break;
-        s = product(Ws_codes, Ws_alpha, vocab, H, k_s, ws.hcodes, ws.hbeta, k_a, bias_s, ws.logits);
+        if (amq::quantized_gemv_supported(H)) {
+            // the quantizer on the new state runs inside the output product's kernel, which also leaves the planes and
+            // coefficients for the recurrent product of the next token
+            s = amq::launch_quantized_gemv(Ws_codes, Ws_alpha, vocab, H, k_s, h, k_a, T, bias_s, ws.logits, ws.hcodes, ws.hbeta,
+                                           st, true);
+        } else {
+            s = amq::launch_quantize(h, H, H, nullptr, 0, 0, 1, k_a, T, ws.hcodes, ws.hbeta, st, true);
+            if (s != AMQ_OK) break;
+            s = product(Ws_codes, Ws_alpha, vocab, H, k_s, ws.hcodes, ws.hbeta, k_a, bias_s, ws.logits);
+        }
         if (s != AMQ_OK) break;
         s = amq::launch_log_softmax_argmax(ws.logits, 1, vocab, vocab, logp ? logp + (size_t)t * vocab : nullptr, vocab,
                                            tokens + t + 1, st, true);

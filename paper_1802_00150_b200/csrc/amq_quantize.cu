@@ -51,7 +51,7 @@ quantize_rows_consecutive_kernel(const float* __restrict__ x, int ldx, int rows,
     }
     float alpha[K];
     uint32_t bits[K];
-    quantize_group<K, 32, 1>(w, valid, n, T, alpha, bits, scratch[warp]);
+    quantize_group<K, 32, 1>(w, valid, n, quant_padding_consecutive(n, 32), T, alpha, bits, scratch[warp]);
     const int wpr = 4 * ((n + 127) / 128);
     if (lane < wpr) {
 #pragma unroll
@@ -65,7 +65,12 @@ quantize_rows_consecutive_kernel(const float* __restrict__ x, int ldx, int rows,
     }
 }
 
-// K bits, EPT elements per thread.  MULTI: one row per CTA (blockDim.x <= 256 threads); else one row per warp.
+// K bits, EPT elements per thread.
+// MULTI: one row per CTA; thread g owns the EPT CONSECUTIVE elements g * EPT .. g * EPT + EPT - 1 (EPT = 8 with 256
+// threads, or 32), so the sign bits the quantizer leaves in a register are a byte (a word) of the packed plane and are
+// stored as such, without a ballot transposition.  The fused matrix-vector kernel quantizes a vector with the same
+// ownership, thread count and summation order, so both leave the same bits.
+// Otherwise one row per warp, lane l owning the elements j * 32 + l.
 template <int K, int EPT, bool MULTI>
 __global__ void __launch_bounds__(256)
 quantize_kernel(RowSource src, int rows, int n, int T, uint32_t* __restrict__ codes, float* __restrict__ coeffs)
@@ -76,27 +81,61 @@ quantize_kernel(RowSource src, int rows, int n, int T, uint32_t* __restrict__ co
     grid_dependency_wait();             // launched early behind a product kernel: its state output must be complete
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int G = MULTI ? blockDim.x : 32;
     const int g = MULTI ? threadIdx.x : lane;
     const int row = MULTI ? blockIdx.x : blockIdx.x * (blockDim.x >> 5) + warp;
     if (row >= rows) return;          // whole group leaves together (row is uniform across the group)
 
     float w[EPT];
     uint32_t valid = 0;
+    if (MULTI) {
+        const int t0 = g * EPT;
+        // whole 16-byte pieces of one source where the addresses allow, single elements otherwise
 #pragma unroll
-    for (int j = 0; j < EPT; ++j) {
-        const int t = j * G + g;
-        const bool ok = t < n;
-        w[j] = ok ? load_elem(src, row, t) : 0.0f;
-        valid |= (ok ? 1u : 0u) << j;
+        for (int q = 0; q < EPT / 4; ++q) {
+            const int t = t0 + 4 * q;
+            const float* p = (t < src.n0) ? src.src0 + (size_t)row * src.ld0 + t : src.src1 + (size_t)row * src.ld1 + (t - src.n0);
+            const bool one_piece = t + 3 < n && (t + 3 < src.n0 || t >= src.n0) && (reinterpret_cast<uintptr_t>(p) & 15u) == 0;
+            if (one_piece) {
+                const float4 v = __ldcg(reinterpret_cast<const float4*>(p));
+                w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+                valid |= 0xFu << (4 * q);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const bool ok = t + e < n;
+                    w[4 * q + e] = ok ? load_elem(src, row, t + e) : 0.0f;
+                    valid |= (ok ? 1u : 0u) << (4 * q + e);
+                }
+            }
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < EPT; ++j) {
+            const int t = j * 32 + g;
+            const bool ok = t < n;
+            w[j] = ok ? load_elem(src, row, t) : 0.0f;
+            valid |= (ok ? 1u : 0u) << j;
+        }
     }
 
     float alpha[K];
     uint32_t bits[K];
-    quantize_group<K, EPT, NW>(w, valid, n, T, alpha, bits, scratch[MULTI ? 0 : warp]);
+    quantize_group<K, EPT, NW>(w, valid, n, MULTI ? quant_padding_consecutive(n, EPT) : quant_padding_strided32(n, EPT), T,
+                               alpha, bits, scratch[MULTI ? 0 : warp]);
 
     const int wpr = 4 * ((n + 127) / 128);
-    pack_group<K, EPT>(bits, lane, MULTI ? warp : 0, G >> 5, wpr, codes + (size_t)row * K * wpr);
+    if (MULTI) {
+        if (g * EPT < wpr * 32) {       // this thread's bits lie inside the plane (zeros past the end of the vector)
+#pragma unroll
+            for (int i = 0; i < K; ++i) {
+                uint32_t* plane = codes + ((size_t)row * K + i) * wpr;
+                if (EPT == 8) reinterpret_cast<uint8_t*>(plane)[g] = (uint8_t)bits[i];
+                else plane[g] = bits[i];
+            }
+        }
+    } else {
+        pack_group<K, EPT>(bits, lane, 0, 1, wpr, codes + (size_t)row * K * wpr);
+    }
     if (g < K) {
         float a = alpha[0];
 #pragma unroll
@@ -145,8 +184,7 @@ amq_status dispatch(const RowSource& src, int rows, int n, int T, uint32_t* code
         const int threads = 32 * ((n128 / 32 + 31) / 32);      // 32 elements per thread
         return run<K, 32, true>(src, rows, n, T, codes, coeffs, threads, st);
     }
-    const int threads = 32 * ((n128 / 8 + 31) / 32);           // 8 elements per thread, up to 256 threads
-    return run<K, 8, true>(src, rows, n, T, codes, coeffs, threads, st);
+    return run<K, 8, true>(src, rows, n, T, codes, coeffs, 256, st);     // 8 elements per thread, always 256 threads
 }
 
 }  // namespace

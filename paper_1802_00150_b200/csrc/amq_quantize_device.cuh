@@ -15,6 +15,9 @@
 // Elements past the end of the vector are zeros that take part in every loop unmasked: their bits are
 // cleared at the end, they add nothing to B^T w, the Gram matrix is counted on masked words, and their known
 // contribution to the greedy |r| sums (all of them follow the trajectory of a zero element) is subtracted.
+// Threads that hold no element of the vector at all leave their |r| sums out instead, so that what is
+// subtracted stays a few elements' worth whatever the size of the group (the subtraction of a large known
+// sum from a rounded one would cost accuracy on short vectors).
 //
 // Arithmetic: sums over the vector are fp32 (per thread, then a fixed butterfly over the warp, then the
 // per-warp partials in a fixed tree, so results are reproducible run to run); the Gram matrix B^T B is exact
@@ -289,8 +292,13 @@ __device__ __forceinline__ int bst_leaf(float x, const float (&thr)[(1 << K) - 1
     return (c1 ? 8 : 0) + (c2 ? 4 : 0) + (c3 ? 2 : 0) + (c4 ? 1 : 0);
 }
 
+// Elements past the end of the vector inside the threads that do hold some of it, for the two ownership patterns in
+// use: thread g owns the EPT consecutive elements from g * EPT; lane l of a warp owns the elements j * 32 + l.
+__host__ __device__ inline int quant_padding_consecutive(int n, int ept) { return (n + ept - 1) / ept * ept - n; }
+__host__ __device__ inline int quant_padding_strided32(int n, int ept) { return (n >= 32 ? 32 : n) * ept - n; }
+
 // Quantize the vector held in w[] (positions past the end of the vector must hold 0 and have their bit
-// clear in `valid`).  NW = 1: the group is the calling warp; NW > 1: the group is the whole CTA of up to NW
+// clear in `valid`; `pad_elems` = how many such positions lie in threads whose `valid` is not zero).  NW = 1: the group is the calling warp; NW > 1: the group is the whole CTA of up to NW
 // warps (quant_scratch_init must have run).  On return alpha[i] are the coefficients and bit j of bits[i] is
 // the sign (1 = +1) of element j of this thread in plane i.
 //
@@ -303,7 +311,7 @@ __device__ __forceinline__ int bst_leaf(float x, const float (&thr)[(1 << K) - 1
 // only): which half of the double-buffered partial-sum scratch the first reduction uses, updated on return,
 // so that consecutive calls keep alternating.
 template <int K, int EPT, int NW>
-__device__ __forceinline__ void quantize_group(const float (&w_in)[EPT], uint32_t valid, int n, int T,
+__device__ __forceinline__ void quantize_group(const float (&w_in)[EPT], uint32_t valid, int n, int pad_elems, int T,
                                                float (&alpha)[K], uint32_t (&bits)[K], QuantScratch<K, NW>& sc,
                                                int* flag = nullptr, int* parity_io = nullptr)
 {
@@ -314,7 +322,8 @@ __device__ __forceinline__ void quantize_group(const float (&w_in)[EPT], uint32_
     const int slot = NW > 1 ? (int)(threadIdx.x >> 5) : 0;
     const int nvalid = __popc(valid);
     const float inv_n = 1.0f / (float)n;
-    const float padding = (float)((NW > 1 ? (int)blockDim.x : 32) * EPT - n);    // zero elements past the end
+    const float padding = (float)pad_elems;                      // zero elements past the end that are summed along
+    const bool holds_some = valid != 0;
     int parity = parity_io ? *parity_io : 0;
 
     float w[EPT];
@@ -341,6 +350,7 @@ __device__ __forceinline__ void quantize_group(const float (&w_in)[EPT], uint32_
             }
             bits[i] = ~neg & valid;
             csum[i] = cs;
+            part = holds_some ? part : 0.0f;
             if (i == K - 1 && T > 0) { last_abs = part; alpha[i] = 0.0f; break; }
             float tot[1] = {part};
             int none[1] = {0};

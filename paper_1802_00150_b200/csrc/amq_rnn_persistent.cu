@@ -236,7 +236,7 @@ rnn_persistent_kernel(PersistArgs a)
         // ---- 2. on-line quantization of z (Algorithm 2); its first barrier also takes the give-up vote ----
         float beta[KA];
         uint32_t bits[KA];
-        quantize_group<KA, EPT, NW>(w, valid, n, a.T, beta, bits, *scratch, &gave_up, &parity);
+        quantize_group<KA, EPT, NW>(w, valid, n, quant_padding_consecutive(n, EPT), a.T, beta, bits, *scratch, &gave_up, &parity);
         if (gave_up) {                                 // uniform over the CTA: leave together
             if (tid == 0) atomicExch(a.status, 1u);
             return;

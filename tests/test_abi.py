@@ -170,3 +170,30 @@ def test_argument_validation_of_the_give_up_selftest(lib):
     assert st(*bad) == -1                                                  # h_last == h0
     bad = list(ok_args); bad[10] = 5
     assert st(*bad) == -2                                                  # bits
+
+
+def test_argument_validation_of_the_one_launch_matrix_vector_entry(lib):
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    fake, odd = vp(0x1000), vp(0x1004)
+    qg = lib.amq_quantized_gemv
+    qg.argtypes = [vp, vp, ci, ci, ci, vp, ci, ci, vp, vp, vp, vp, vp]
+    assert qg(fake, fake, 8, 2049, 2, fake, 2, 2, None, fake, None, None, None) == -2      # vector too long for the fused form
+    assert qg(fake, fake, 8, 64, 5, fake, 2, 2, None, fake, None, None, None) == -2        # bits
+    assert qg(fake, fake, 8, 64, 2, fake, 2, -1, None, fake, None, None, None) == -2       # cycles
+    assert qg(fake, fake, 8, 0, 2, fake, 2, 2, None, fake, None, None, None) == -1         # empty vector
+    assert qg(fake, fake, 8, 64, 2, None, 2, 2, None, fake, None, None, None) == -1        # no vector
+    assert qg(odd, fake, 8, 64, 2, fake, 2, 2, None, fake, None, None, None) == -3
+    assert qg(fake, fake, 8, 64, 2, fake, 2, 2, None, fake, odd, None, None) == -3
+    assert qg(None, None, 0, 64, 2, None, 2, 2, None, None, None, None, None) == 0         # no rows: nothing to do
+
+
+def test_paper_table6_fixture_is_the_one_the_benchmark_reads():
+    """bench.py quotes the paper's single-core CPU times (Appendix A, Table 6) from this fixture: the four quantized rows
+    must be there with the printed totals."""
+    rows = {}
+    for ln in open(os.path.join(ROOT, "tests", "golden", "table6_cpu_ms.txt")):
+        f = ln.split()
+        if len(f) >= 6 and f[0].isdigit():
+            rows[(int(f[0]), int(f[2]))] = float(f[4])
+    assert rows[(4096, 2)] == 0.35 and rows[(4096, 3)] == 0.72 and rows[(42000, 2)] == 3.17 and rows[(42000, 3)] == 6.46
+    assert rows[(4096, 0)] == 1.95 and rows[(42000, 0)] == 19.10       # the full-precision baseline of the same table

@@ -449,3 +449,45 @@ def test_batched_sequences_repeat_bit_for_bit(amq, cell, I, H, kw, ka, batch, st
         del junk
     for r in runs[1:]:
         assert torch.equal(r, runs[0])
+
+
+@pytest.mark.parametrize("m,n,kw,ka,T", [(4096, 1024, 2, 2, 2), (1000, 1024, 3, 3, 2), (300, 2048, 2, 3, 2), (77, 600, 4, 4, 2),
+                                         (513, 100, 1, 2, 3), (64, 1, 2, 2, 2), (35, 2047, 3, 1, 0), (42000, 1024, 2, 2, 2)])
+def test_quantized_gemv_in_one_launch(amq, m, n, kw, ka, T):
+    """Table 6's operation (on-line quantization of one vector + binary matrix-vector product) as a single launch: the
+    vector's planes and coefficients against the oracle under the staged protocol, the product against the oracle on
+    those planes, and both bit for bit against the two-call path (same ownership and summation order by design)."""
+    W = synth.normal((m, n), 0.03, 400 + m, 1).astype(np.float64)
+    x = synth.uniform((1, n), -1, 1, 400 + m, 2)
+    bias = synth.normal((m,), 0.1, 400 + m, 3)
+    Wc, Wa = oracle.quantize_rows(W, kw, 2)
+    dWc, dWa = codes_dev(Wc), dev(Wa, torch.float32)
+
+    def fused_quantizer(a, k, stage):
+        _, xc, xb = amq.quantized_gemv(dWc[:8].contiguous(), dWa[:8].contiguous(), dev(a[0]), k, stage, want_codes=True)
+        torch.cuda.synchronize()
+        return codes_np(xc)[None], xb.cpu().numpy()[None]
+
+    print(parity.compare_quantizer(x, ka, T, fused_quantizer))
+    y, xc, xb = amq.quantized_gemv(dWc, dWa, dev(x[0]), ka, T, bias=dev(bias), want_codes=True)
+    ref = oracle.binary_gemm(Wc, Wa, codes_np(xc)[None], xb.cpu().numpy().astype(np.float64)[None], n, bias.astype(np.float64))
+    assert np.abs(y.cpu().numpy() - ref[0]).max() <= 1e-5 * (np.abs(ref).max() + 1)
+    o_xc, o_xb = oracle.quantize_rows(x.astype(np.float64), ka, T)
+    full = oracle.binary_gemm(Wc, Wa, o_xc, o_xb, n, bias.astype(np.float64))
+    if np.array_equal(o_xc, codes_np(xc)[None]):
+        assert np.all(np.abs(y.cpu().numpy() - full[0]) <= parity.output_tolerance(Wa, o_xb, n)[0] + 1e-6)
+    # the two-call path leaves the same bits
+    c2, b2 = amq.quantize(dev(x), ka, T)
+    assert torch.equal(c2[0], xc) and torch.equal(b2[0], xb)
+    y2 = amq.binary_gemm(dWc, dWa, c2, b2, n, bias=dev(bias))
+    assert torch.equal(y2[0], y)
+    # repeatable
+    y3 = amq.quantized_gemv(dWc, dWa, dev(x[0]), ka, T, bias=dev(bias))
+    assert torch.equal(y3, y)
+
+
+def test_quantized_gemv_rejects_long_vectors(amq):
+    Wc, Wa = oracle.quantize_rows(synth.normal((8, 2049), 0.03, 9, 1).astype(np.float64), 2, 2)
+    with pytest.raises(amq.AmqError) as e:
+        amq.quantized_gemv(codes_dev(Wc), dev(Wa, torch.float32), dev(synth.uniform((2049,), -1, 1, 9, 2)), 2, 2)
+    assert e.value.status == -2
