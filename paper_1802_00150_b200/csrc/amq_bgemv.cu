@@ -44,6 +44,9 @@ struct GemvParams {
 
 constexpr int FQ_EPT = 8;       // fused form: 256 threads x 8 consecutive elements each
 constexpr int FQ_MAX_CH = 16;   // = 2048 bit positions
+#ifndef FQ_CTAS_PER_SM
+#define FQ_CTAS_PER_SM 1
+#endif
 
 // differing bits of (w xor x) over the four words of a chunk, accumulated carry-save:
 // `ones` carries the bit-wise sums, the return value counts the carries (weight 2)
@@ -248,7 +251,7 @@ amq_status launch_cfg(const GemvParams& p, cudaStream_t st)
     constexpr int R = R0 < SEG ? R0 : SEG;
     const bool exact = p.CH == CPT * SEG;
     auto kernel = exact ? bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, true, FQ> : bgemv_kernel<KW, KA, CPT, R, SEG_LOG2, false, FQ>;
-    static thread_local int cached_dev = -1, cached_grid[2] = {0, 0};
+    static thread_local int cached_dev = -1, cached_grid[2] = {0, 0}, cached_sms = 0;
     int dev = 0;
     AMQ_CUDA_TRY(cudaGetDevice(&dev));
     if (dev != cached_dev) {
@@ -261,11 +264,14 @@ amq_status launch_cfg(const GemvParams& p, cudaStream_t st)
             cached_grid[e] = sms * (per_sm > 0 ? per_sm : 1);
         }
         cached_dev = dev;
+        cached_sms = sms;
     }
     constexpr int PASSES = SEG / R;
     const long long passes = ((long long)p.m + 31) / 32 * PASSES;
     const long long need = (passes + 7) / 8;                            // small matrices: one pass per warp, spread over the SMs
-    const int limit = cached_grid[exact ? 1 : 0];
+    // fused form: every CTA repeats the quantization, so no more than FQ_CTAS_PER_SM of them share an SM's issue slots
+    const int limit = FQ ? (cached_sms * FQ_CTAS_PER_SM < cached_grid[exact ? 1 : 0] ? cached_sms * FQ_CTAS_PER_SM : cached_grid[exact ? 1 : 0])
+                         : cached_grid[exact ? 1 : 0];
     const int grid = (int)(need < limit ? need : limit);
     AMQ_CUDA_TRY(launch_kernel(kernel, dim3((unsigned)grid), dim3(256), 0, st, p.overlap, p));
     AMQ_LAUNCH_CHECK();

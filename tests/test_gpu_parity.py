@@ -491,3 +491,31 @@ def test_quantized_gemv_rejects_long_vectors(amq):
     with pytest.raises(amq.AmqError) as e:
         amq.quantized_gemv(codes_dev(Wc), dev(Wa, torch.float32), dev(synth.uniform((2049,), -1, 1, 9, 2)), 2, 2)
     assert e.value.status == -2
+
+
+@pytest.mark.parametrize("batch", [1, 6])
+def test_two_stacked_layers(amq, batch):
+    """Stacking: the h sequence of one layer is the x sequence of the next, handed over on the device.  The second layer
+    is held against the oracle run on the very sequence the first layer produced (first step within the state tolerance,
+    the free-running rest within the drift bound of the other sequence tests); LSTM below a GRU to cover both cells."""
+    I, H1, H2, steps, ka = 48, 64, 40, 5, 2
+    W1c, W1a, b1 = cell_setup("lstm", I, H1, 2, 301, 0.08)
+    W2c, W2a, b2 = cell_setup("gru", H1, H2, 3, 302, 0.08)
+    xs = synth.normal((steps, batch, I), 1.0, 303, 1)
+    z1 = np.zeros((batch, H1), dtype=np.float32)
+    z2 = np.zeros((batch, H2), dtype=np.float32)
+    ws1 = amq.new_workspace(I, H1, batch, ka)
+    ws2 = amq.new_workspace(H1, H2, batch, ka)
+    seq1, _, _ = amq.lstm_sequence(codes_dev(W1c), dev(W1a, torch.float32), dev(b1), I, H1, dev(xs), dev(z1), dev(z1), ka, 2, ws1,
+                                   want_h_seq=True)
+    seq2, last2 = amq.gru_sequence(codes_dev(W2c), dev(W2a, torch.float32), dev(b2), H1, H2, seq1, dev(z2), ka, 2, ws2,
+                                   want_h_seq=True)
+    assert amq.workspace_status(ws1) == 0 and amq.workspace_status(ws2) == 0
+    o1, _, _ = oracle.lstm_sequence(W1c, W1a, b1, I, H1, xs, z1, z1, ka, 2)
+    assert np.abs(seq1.cpu().numpy() - o1).max() <= 0.05
+    x2 = seq1.cpu().numpy()
+    o2, o2_last = oracle.gru_sequence(W2c, W2a, b2, H1, H2, x2, z2, ka, 2)
+    _, beta = oracle.quantize_rows(np.concatenate([x2[0].astype(np.float64), z2], axis=1), ka, 2)
+    assert np.abs(seq2[0].cpu().numpy() - o2[0]).max() <= state_tolerance(W2a, beta, H1 + H2)
+    assert np.abs(seq2.cpu().numpy() - o2).max() <= 0.05
+    assert torch.equal(seq2[-1], last2)
