@@ -307,7 +307,7 @@ AMQ_API amq_status amq_log_softmax_argmax(const float* logits, int rows, int n, 
                                   float* logp, int ldp, int32_t* argmax, void* stream);
 
 /*
- * Greedy decoding with the language model of Eq. 6, one sequence, enqueued as one chain on `stream` (seven kernel
+ * Greedy decoding with the language model of Eq. 6, one sequence, enqueued as one chain on `stream` (six or seven kernel
  * launches per token, no host round trip).  For t = 0 .. steps-1:
  *   x_t = row tokens[t] of the quantized embedding (We_codes [vocab][k_e][wpr(I)], We_alpha [vocab][k_e]);
  *   (h, c) <- LSTM step in the paper's own form (W_i [4H x I], W_h [4H x H], k_w bits, bias [4H] or NULL; h quantized

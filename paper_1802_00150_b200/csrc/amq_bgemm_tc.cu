@@ -219,6 +219,20 @@ __device__ __forceinline__ void expand_chunk(uint32_t base, const uint32_t (&off
 
 __device__ __forceinline__ float logistic(float v) { return 1.0f / (1.0f + __expf(-v)); }
 
+// x / d for x >= 0 and the small divisors that occur in the row bookkeeping (bits per weight 1..4; gates 1, 3, 4): inside the
+// switch the divisor is a constant, so each case is a shift or one multiplication instead of the generic division sequence
+// (every expander thread runs several of these before its first load; they were a visible part of a CTA's start-up time)
+__device__ __forceinline__ int div_small(int x, int d)
+{
+    switch (d) {
+        case 1: return x;
+        case 2: return x >> 1;
+        case 3: return x / 3;
+        case 4: return x >> 2;
+        default: return x / d;
+    }
+}
+
 // Epilogue, first half: tensor memory -> registers -> partial products y[plane-row][batch entry] in shared memory
 // (EPI_DOTS: the integer partials straight to global memory).  A thread is a plane-row (lane of tensor memory, lane
 // quarter `quarter` = warp index mod 4); the work items (M tile, column segment, 8 batch entries = 8 * KA columns)
@@ -237,11 +251,11 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
     const uint32_t tlane = tmem_acc + ((uint32_t)(quarter * 32) << 16);
     if (a.epilogue == EPI_DOTS) {
         const int pad = p.wpr * 32 - a.n;
-        const int l = pr / k_w, i = pr - l * k_w;
-        const int gate = l % p.gates;
+        const int l = div_small(pr, k_w), i = pr - l * k_w;
+        const int lg = div_small(l, p.gates), gate = l - lg * p.gates;
         for (int mt = 0; mt < p.MT; ++mt)                           // (one column segment in this epilogue)
         for (int g = slot; g < groups; g += nslots) {
-            const int u = u0 + mt * p.UT + l / p.gates;
+            const int u = u0 + mt * p.UT + lg;
             const bool row_ok = pr < TMp && u < p.units;
             const size_t row = (size_t)gate * p.units + u;
             int acc[KA][8];
@@ -440,7 +454,7 @@ bgemm_tc_kernel(TcParams p)
     if (warp < mma_warp) {
         // ---- expanders: G groups of EXP threads take the steps in turn; inside a group thread r owns operand
         //      row r (A plane-rows first, then the B rows) ----
-        const int grp = tid / EXP, r_all = tid - grp * EXP;
+        const int grp = (tid >= EXP ? 1 : 0) + (tid >= 2 * EXP ? 1 : 0) + (tid >= 3 * EXP ? 1 : 0), r_all = tid - grp * EXP;   // G <= 4
         const uint4* src = nullptr;
         uint32_t dst0;                                              // shared address of the row in stage 0
         const float* coef_src = nullptr;                            // the row's coefficient, staged for the epilogue
@@ -450,8 +464,9 @@ bgemm_tc_kernel(TcParams p)
             const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
             size_t prow = 0;                                        // plane-row index in Wcodes / Walpha
             if (r < TMp) {
-                const int l = r / k_w, i = r - l * k_w;
-                const int u = u0 + mt * p.UT + l / p.gates, gate = l % p.gates;
+                const int l = div_small(r, k_w), i = r - l * k_w;
+                const int lg = div_small(l, p.gates), gate = l - lg * p.gates;
+                const int u = u0 + mt * p.UT + lg;
                 if (u < p.units) {
                     prow = ((size_t)gate * p.units + u) * k_w + i;
                     src = reinterpret_cast<const uint4*>(a.Wcodes + prow * p.wpr);
@@ -474,6 +489,15 @@ bgemm_tc_kernel(TcParams p)
                 if (j == 0) corr_src = coef_src;
             }
         }
+        // weight rows are fetched at once, before anything else is set up (their latency is the longest item of a
+        // CTA's start-up); everything the preceding kernel of the stream may have written (the activation planes and
+        // their coefficients, the state) is read after the wait
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+        const bool weight_row = r_all < MT * TILE_M;
+        if (!weight_row) grid_dependency_wait();
+        uint4 cur = (src && grp < CH) ? load_row_chunk(src + grp, weight_row) : zero;       // own steps: grp, grp + G, ..
+        uint4 nxt = (src && grp + G < CH) ? load_row_chunk(src + grp + G, weight_row) : zero;
+        if (weight_row) grid_dependency_wait();
         const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
         uint32_t off[8];                                            // swizzled position of chunk j: j xor (row mod 8)
 #pragma unroll
@@ -482,25 +506,16 @@ bgemm_tc_kernel(TcParams p)
 #pragma unroll
         for (int s = 0; s < 7; ++s) mul[s] = p.mul[s];
         const uint32_t m_sign = p.mask_sign, m_half = p.mask_half;  // 0x80808080, 0x40404040
-        const uint4 zero = make_uint4(0, 0, 0, 0);
-
-        // weight rows are fetched at once; everything the preceding kernel of the stream may have written (the
-        // activation planes and their coefficients, the state) is read after the wait
-        const bool weight_row = r_all < MT * TILE_M;
-        if (!weight_row) grid_dependency_wait();
-        uint4 cur = (src && grp < CH) ? load_row_chunk(src + grp, weight_row) : zero;       // own steps: grp, grp + G, ..
-        uint4 nxt = (src && grp + G < CH) ? load_row_chunk(src + grp + G, weight_row) : zero;
-        if (weight_row) grid_dependency_wait();
-        // coefficients for the epilogue, after the first operand loads are under way (the stores below wait for
-        // their loads; the latency hides behind the main loop)
-        if (coef_dst) {
-            *coef_dst = coef_src ? __ldcg(coef_src) : 0.0f;
-            if (r_all >= MT * TILE_M && (r_all - MT * TILE_M) % KA == 0) {
-                float sum = 0.0f;
-                for (int jj = 0; jj < KA; ++jj) sum += corr_src ? __ldcg(corr_src + jj) : 0.0f;
-                sBcorr[(r_all - MT * TILE_M) / KA] = -(float)(p.wpr * 32 - a.n) * sum;
-            }
+        // coefficients for the epilogue: the loads are issued now, after the first operand loads, and their values are
+        // stored only after this thread's first pipeline step, so that no thread waits for them before it has work out
+        float coef_val = 0.0f, corr_sum = 0.0f;
+        const bool has_corr = coef_dst && r_all >= MT * TILE_M && (r_all - MT * TILE_M) % KA == 0;
+        if (coef_dst && coef_src) coef_val = __ldcg(coef_src);
+        if (has_corr && corr_src) {
+#pragma unroll
+            for (int jj = 0; jj < KA; ++jj) corr_sum += __ldcg(corr_src + jj);
         }
+        bool coef_pending = coef_dst != nullptr;
         int buf = grp;                                              // G <= S
         uint32_t empty_parity = 1;                                  // parity that means "never used" on the first lap
         for (int c = grp; c < CH; c += G) {
@@ -514,8 +529,17 @@ bgemm_tc_kernel(TcParams p)
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
+            if (coef_pending) {
+                *coef_dst = coef_val;
+                if (has_corr) sBcorr[(r_all - MT * TILE_M) / KA] = -(float)(p.wpr * 32 - a.n) * corr_sum;
+                coef_pending = false;
+            }
             buf += G;
             if (buf >= S) { buf -= S; empty_parity ^= 1u; }
+        }
+        if (coef_pending) {                                         // (a group without a step of its own)
+            *coef_dst = coef_val;
+            if (has_corr) sBcorr[(r_all - MT * TILE_M) / KA] = -(float)(p.wpr * 32 - a.n) * corr_sum;
         }
     } else if (lane == 0) {
         // ---- MMA issuer ----
@@ -636,16 +660,16 @@ bgemm_tc_persistent_kernel(TcParams p)
     if (warp < mma_warp) {
         // ---- expanders: thread r of a group owns operand row r of every tile; the groups take the steps of the
         //      CTA's whole sequence (tiles x steps per tile) in turn ----
-        const int grp = tid / EXP, r_all = tid - grp * EXP;
+        const int grp = (tid >= EXP ? 1 : 0) + (tid >= 2 * EXP ? 1 : 0) + (tid >= 3 * EXP ? 1 : 0), r_all = tid - grp * EXP;   // G <= 4
         const bool is_a = r_all < MT * TILE_M;
         int unit_off = 0, gate = 0, plane = 0, entry = 0;
         bool valid;
         uint32_t dst0;
         if (is_a) {
             const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
-            const int l = r / k_w;
+            const int l = div_small(r, k_w), lg = div_small(l, p.gates);
             valid = r < TMp;
-            plane = r - l * k_w; unit_off = mt * p.UT + l / p.gates; gate = l % p.gates;
+            plane = r - l * k_w; unit_off = mt * p.UT + lg; gate = l - lg * p.gates;
             dst0 = smem_u32(stage_base) + r_all * 128;
         } else {
             const int r = r_all - MT * TILE_M;
@@ -754,8 +778,9 @@ bgemm_tc_persistent_kernel(TcParams p)
             if (a.epilogue != EPI_DOTS) {
                 for (int idx = tid_e; idx < MT * TILE_M; idx += nth_e) {
                     const int mt = idx >> 7, r = idx & (TILE_M - 1);
-                    const int l = r / k_w, i = r - l * k_w;
-                    const int u = u0 + mt * p.UT + l / p.gates, gate = l % p.gates;
+                    const int l = div_small(r, k_w), i = r - l * k_w;
+                    const int lg = div_small(l, p.gates);
+                    const int u = u0 + mt * p.UT + lg, gate = l - lg * p.gates;
                     sAlpha[idx] = (r < TMp && u < p.units) ? __ldg(a.Walpha + ((size_t)gate * p.units + u) * k_w + i) : 0.0f;
                 }
                 for (int idx = tid_e; idx < n_mma; idx += nth_e) {

@@ -79,7 +79,7 @@ amq_status recurrent_part(const PaperCall& c, const PaperWorkspace& ws, const fl
     // in a sequence the kernel before this quantizer is the recurrent product of the previous timestep: when that
     // runs as a single wave the quantizer may be scheduled behind it early (it waits for it first thing)
     // (with one sequence every kernel of the step is short and waits for its predecessor first thing: all overlapped)
-    if (c.batch == 1 && quantized_gemv_supported(c.H)) {
+    if (c.batch == 1 && quantized_gemv_supported(c.H) && c.k_a <= 2) {
         // one sequence, a state of up to 2048 elements: the quantizer runs inside the matrix-vector kernel (one launch
         // for both; the same bits as the two launches below), then the small gate kernel
         amq_status s1 = launch_quantized_gemv(c.Wh_codes, c.Wh_alpha, 4 * c.H, c.H, c.k_w, h_in, c.k_a, c.T, nullptr, ws.gates,

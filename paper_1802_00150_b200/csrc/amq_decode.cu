@@ -3,7 +3,8 @@
 // the input projection W_i x + b, the recurrent product W_h h_hat on the on-line quantized state, the gates, the
 // quantizer on the new state (its planes serve the output layer now and the recurrence of the next token), the
 // output product W_s h_hat + b_s and log-softmax / arg-max.  Six launches per token (the quantizer on the new state
-// runs inside the output product's kernel when the state has at most 2048 elements, else seven), no host round trip.
+// runs inside the output product's kernel when the state has at most 2048 elements and at most 2 bits, else seven), no
+// host round trip.
 #include "amq_common.cuh"
 
 namespace amq {
@@ -89,7 +90,7 @@ amq_status amq_lm_greedy_decode(const uint32_t* We_codes, const float* We_alpha,
         if (s != AMQ_OK) break;
         s = amq::launch_lstm_gates(ws.pre, ws.proj, c, h, c, H, st, true);                  // state updated in place
         if (s != AMQ_OK) break;
-        if (amq::quantized_gemv_supported(H)) {
+        if (amq::quantized_gemv_supported(H) && k_a <= 2) {       // (with more planes the repeated k x k solves cost more than a launch)
             // the quantizer on the new state runs inside the output product's kernel, which also leaves the planes and
             // coefficients for the recurrent product of the next token
             s = amq::launch_quantized_gemv(Ws_codes, Ws_alpha, vocab, H, k_s, h, k_a, T, bias_s, ws.logits, ws.hcodes, ws.hbeta,
