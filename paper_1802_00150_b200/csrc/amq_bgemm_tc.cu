@@ -160,6 +160,43 @@ __device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t
         :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// The four MMAs of one pipeline stage (K = 4 x 32 bytes of the same swizzled rows) into one accumulator, as one block:
+// the two descriptors are rebuilt from their low words (the high words are the same constant for both operands; the
+// start-address field advances by 32 bytes = 2 units per MMA and cannot carry out of its 14 bits below 256 KiB), so the
+// single issuing thread spends a dozen instructions per stage instead of several per MMA: its pace, not the tensor
+// pipe's, was what a stage cost.  `acc_first`: whether the first of the four accumulates (the other three always do).
+__device__ __forceinline__ void mma_i8_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                             uint32_t acc_first)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .b64 da, db;\n\t"
+        ".reg .b32 al, bl;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "setp.eq.b32 q, %5, %5;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t"
+        "add.u32 al, %1, 2;\n\t"
+        "add.u32 bl, %2, 2;\n\t"
+        "mov.b64 da, {al, %3};\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, q;\n\t"
+        "add.u32 al, %1, 4;\n\t"
+        "add.u32 bl, %2, 4;\n\t"
+        "mov.b64 da, {al, %3};\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, q;\n\t"
+        "add.u32 al, %1, 6;\n\t"
+        "add.u32 bl, %2, 6;\n\t"
+        "mov.b64 da, {al, %3};\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, q;\n\t"
+        "}"
+        :: "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc_first) : "memory");
+}
+
 __device__ __forceinline__ void mma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
@@ -553,14 +590,26 @@ bgemm_tc_kernel(TcParams p)
             // descriptors of the stage: start addresses are below 256 KiB, so adding to the low word never carries
             const uint64_t adesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
             const uint64_t bdesc0 = adesc0 + (uint64_t)(a_stage_bytes >> 4);
-#pragma unroll
-            for (int qq = 0; qq < STAGE_WORDS; ++qq) {
-                const int word = c * STAGE_WORDS + qq;
-                const int seg = word >= split_word ? 1 : 0;
-                const uint32_t accumulate = (word != 0 && word != split_word) ? 1u : 0u;
-                mma_i8(tmem_base + seg * n_mma, adesc0 + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+            const int word0 = c * STAGE_WORDS;
+            if (word0 >= split_word || word0 + STAGE_WORDS <= split_word) {
+                // the whole stage lies in one column segment (always, unless a GRU's input width is not a multiple of 128)
+                const int seg = word0 >= split_word ? 1 : 0;
+                const uint32_t acc_first = (word0 != 0 && word0 != split_word) ? 1u : 0u;
+                const uint32_t hi = (uint32_t)(desc_base >> 32);
+                mma_i8_stage(tmem_base + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first);
                 if (MT == 2)
-                    mma_i8(tmem_base + (p.nseg + seg) * n_mma, adesc0 + (TILE_M * 128 >> 4) + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                    mma_i8_stage(tmem_base + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi, idesc,
+                                 acc_first);
+            } else {
+#pragma unroll
+                for (int qq = 0; qq < STAGE_WORDS; ++qq) {
+                    const int word = word0 + qq;
+                    const int seg = word >= split_word ? 1 : 0;
+                    const uint32_t accumulate = (word != 0 && word != split_word) ? 1u : 0u;
+                    mma_i8(tmem_base + seg * n_mma, adesc0 + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                    if (MT == 2)
+                        mma_i8(tmem_base + (p.nseg + seg) * n_mma, adesc0 + (TILE_M * 128 >> 4) + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                }
             }
             mma_commit(smem_u32(&empty_bar[buf]));
             if (++buf == S) { buf = 0; full_parity ^= 1u; }
@@ -747,14 +796,25 @@ bgemm_tc_persistent_kernel(TcParams p)
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t adesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
                     const uint64_t bdesc0 = adesc0 + (uint64_t)(a_stage_bytes >> 4);
-#pragma unroll
-                    for (int qq = 0; qq < STAGE_WORDS; ++qq) {
-                        const int word = c * STAGE_WORDS + qq;
-                        const int seg = word >= split_word ? 1 : 0;
-                        const uint32_t accumulate = (word != 0 && word != split_word) ? 1u : 0u;
-                        mma_i8(acc + seg * n_mma, adesc0 + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                    const int word0 = c * STAGE_WORDS;
+                    if (word0 >= split_word || word0 + STAGE_WORDS <= split_word) {
+                        const int seg = word0 >= split_word ? 1 : 0;
+                        const uint32_t acc_first = (word0 != 0 && word0 != split_word) ? 1u : 0u;
+                        const uint32_t hi = (uint32_t)(desc_base >> 32);
+                        mma_i8_stage(acc + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first);
                         if (MT == 2)
-                            mma_i8(acc + (p.nseg + seg) * n_mma, adesc0 + (TILE_M * 128 >> 4) + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                            mma_i8_stage(acc + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi, idesc,
+                                         acc_first);
+                    } else {
+#pragma unroll
+                        for (int qq = 0; qq < STAGE_WORDS; ++qq) {
+                            const int word = word0 + qq;
+                            const int seg = word >= split_word ? 1 : 0;
+                            const uint32_t accumulate = (word != 0 && word != split_word) ? 1u : 0u;
+                            mma_i8(acc + seg * n_mma, adesc0 + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                            if (MT == 2)
+                                mma_i8(acc + (p.nseg + seg) * n_mma, adesc0 + (TILE_M * 128 >> 4) + 2 * qq, bdesc0 + 2 * qq, idesc, accumulate);
+                        }
                     }
                     mma_commit(smem_u32(&empty_bar[buf]));
                     if (++buf == S) { buf = 0; full_parity ^= 1u; }
