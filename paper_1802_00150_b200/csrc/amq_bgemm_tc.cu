@@ -1,5 +1,5 @@
-// Batched binary matrix product on the 5th-generation tensor cores (tcgen05.mma kind::i8, accumulators
-// in tensor memory), in the stacked form of Fig. 3, right: the k_w planes of the weight rows of a tile are
+// Batched binary matrix product on the 5th-generation tensor cores (tcgen05.mma kind::i8 or kind::mxf4,
+// accumulators in tensor memory), in the stacked form of Fig. 3, right: the k_w planes of the weight rows of a tile are
 // the M rows of one integer matrix product, the k_a planes of the activation vectors its N columns, the
 // packed bit positions its K dimension; the k_w x k_a partials of every (row, vector) pair are folded
 // with the row-wise coefficients afterwards (Sec. 4), and for the cells the gate arithmetic of Eq. 6 /
@@ -14,6 +14,13 @@
 // both operands, which a dot product does not see.  What bounds the main loop is the shared-memory port, which
 // the expansion stores (128 operand bytes per row and stage) share with the operand reads of the MMAs
 // (an M 128 x N 256 x K 32 instruction reads 12 KB), not the arithmetic.
+//
+// Where tensor memory has 16 columns left beside the accumulators, the operands are 4-bit instead (kind::mxf4, block
+// scaled): bit 1 -> the E2M1 nibble 0xA (-1.0), bit 0 -> 0x2 (+1.0), one shift-and-mask per eight nibbles; the block
+// scales (one E8M0 byte per 32 elements, read from tensor memory) are all 2^0, the accumulators fp32, exact for sums
+// of +-1 up to 2^24 terms.  The same 128 bytes of a row then hold 256 bit positions: half the shared-memory traffic
+// and half the MMA time per bit position.  Not possible where the accumulators fill all 512 columns (two M tiles at
+// N = 256).
 //
 // Shared-memory operand layout: K-major with the 128-byte swizzle: a pipeline stage holds 128 bytes of K per
 // operand row, rows are 128 bytes apart, groups of 8 rows 1024 bytes apart, and the 16-byte chunk j of row r
@@ -74,6 +81,13 @@ struct TcParams {
     // issue on the FMA pipe) and its two byte masks (so that one LOP3 takes both from registers)
     uint32_t mul[8];
     uint32_t mask_sign, mask_half;
+    // 4-bit operand form (kind::mxf4: bits expanded to E2M1 nibbles +-1, unit block scales, fp32 accumulators): a pipeline
+    // stage then holds 256 bit positions per row in the same 128 bytes, i.e. half the shared-memory traffic and half the
+    // MMA time per bit position.  Used when the 16 tensor-memory columns of the scale factors fit beside the accumulators.
+    int fp4;
+    int sf_col;     // first tensor-memory column of the scale factors (all bytes 0x7F = 2^0)
+    int steps;      // pipeline steps per tile: chunks of 128 bit positions, or pairs of them
+    int pad;        // bit positions per row that are zero in both operands (they add +1 each to every dot product)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -254,6 +268,75 @@ __device__ __forceinline__ void expand_chunk(uint32_t base, const uint32_t (&off
     }
 }
 
+// 4-bit form: one 128-bit chunk of a packed row -> its 128 nibbles (64 bytes: four 16-byte pieces at the swizzled offsets
+// off[0..3]).  Bit 1 -> 0xA (-1.0 in E2M1), bit 0 -> 0x2 (+1.0).  Output word s of a packed word keeps its bits s, s + 4, ..,
+// s + 28 in its eight nibbles: the K positions inside a word are permuted, identically for both operands.
+__device__ __forceinline__ void expand_chunk_fp4(uint32_t base, const uint32_t* off, const uint4& v)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint32_t y0 = ((w[q] << 3) & 0x88888888u) | 0x22222222u;
+        const uint32_t y1 = ((w[q] << 2) & 0x88888888u) | 0x22222222u;
+        const uint32_t y2 = ((w[q] << 1) & 0x88888888u) | 0x22222222u;
+        const uint32_t y3 = (w[q] & 0x88888888u) | 0x22222222u;
+        st_shared_v4(base + off[q], y0, y1, y2, y3);
+    }
+}
+
+// The four MMAs of one pipeline stage in the 4-bit form (K = 4 x 64 nibbles = the same 4 x 32 bytes of the swizzled rows),
+// block scales of 32 elements read from tensor memory (all ones), fp32 accumulators.
+__device__ __forceinline__ void mma_mxf4_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                               uint32_t acc_first, uint32_t sf_tmem)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .b64 da, db;\n\t"
+        ".reg .b32 al, bl;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "setp.eq.b32 q, %5, %5;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %4, [%6], [%6], p;\n\t"
+        "add.u32 al, %1, 2;\n\t"
+        "add.u32 bl, %2, 2;\n\t"
+        "mov.b64 da, {al, %3};\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %4, [%6], [%6], q;\n\t"
+        "add.u32 al, %1, 4;\n\t"
+        "add.u32 bl, %2, 4;\n\t"
+        "mov.b64 da, {al, %3};\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %4, [%6], [%6], q;\n\t"
+        "add.u32 al, %1, 6;\n\t"
+        "add.u32 bl, %2, 6;\n\t"
+        "mov.b64 da, {al, %3};\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %4, [%6], [%6], q;\n\t"
+        "}"
+        :: "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc_first), "r"(sf_tmem) : "memory");
+}
+
+// Scale factors of the 4-bit form: 16 tensor-memory columns, every byte 0x7F (2^0 in E8M0), written by four warps (one per
+// lane quarter); both operands' scale addresses point at this region, whose every byte is the same.
+__device__ __forceinline__ void write_unit_scales(uint32_t tmem_base, int sf_col, int warp)
+{
+    const uint32_t t = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)sf_col;
+    const uint32_t one = 0x7F7F7F7Fu;
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+        :: "r"(t), "r"(one) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+
+// an accumulator as the epilogue reads it from tensor memory -> the exact integer dot product (pad positions included)
+__device__ __forceinline__ float acc_to_float(int acc, bool fp4)
+{
+    return fp4 ? __int_as_float(acc) : small_int_to_float(acc >> 12);
+}
+
 __device__ __forceinline__ float logistic(float v) { return 1.0f / (1.0f + __expf(-v)); }
 
 // x / d for x >= 0 and the small divisors that occur in the row bookkeeping (bits per weight 1..4; gates 1, 3, 4): inside the
@@ -287,7 +370,8 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
     const int groups = p.TB >> 3;
     const uint32_t tlane = tmem_acc + ((uint32_t)(quarter * 32) << 16);
     if (a.epilogue == EPI_DOTS) {
-        const int pad = p.wpr * 32 - a.n;
+        const int pad = p.pad;
+        const bool fp4 = p.fp4 != 0;
         const int l = div_small(pr, k_w), i = pr - l * k_w;
         const int lg = div_small(l, p.gates), gate = l - lg * p.gates;
         for (int mt = 0; mt < p.MT; ++mt)                           // (one column segment in this epilogue)
@@ -303,12 +387,14 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
             for (int col = 0; col < 8 * KA; ++col) {
                 const int b = b0 + g * 8 + col / KA;
                 if (row_ok && b < a.batch)
-                    a.D[(((size_t)b * a.m + row) * k_w + i) * KA + col % KA] = (acc[col / 8][col % 8] >> 12) - pad;
+                    a.D[(((size_t)b * a.m + row) * k_w + i) * KA + col % KA] =
+                        (fp4 ? (int)__int_as_float(acc[col / 8][col % 8]) : (acc[col / 8][col % 8] >> 12)) - pad;
             }
         }
         return;
     }
     // loops without divisions: the per-item overhead is spread over only 8 * KA accumulators per thread
+    const bool fp4 = p.fp4 != 0;
     for (int mt = 0; mt < p.MT; ++mt)
     for (int seg = 0; seg < p.nseg; ++seg)
     for (int g = slot; g < groups; g += nslots) {
@@ -339,7 +425,7 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
                     const float4 t = b4[bi >> 2];
                     const float beta = (bi & 3) == 0 ? t.x : (bi & 3) == 1 ? t.y : (bi & 3) == 2 ? t.z : t.w;
                     const int col = (half * 4 + e4) * KA + j;
-                    y += beta * small_int_to_float(acc[col / 8][col % 8] >> 12);
+                    y += beta * acc_to_float(acc[col / 8][col % 8], fp4);
                 }
                 yrow[half * 4 + e4] = alpha * y;
             }
@@ -438,7 +524,7 @@ __device__ __forceinline__ void epilogue_smem_to_global(const TcParams& p, const
     }
 }
 
-template <int KA>
+template <int KA, bool FP4>
 __global__ void __launch_bounds__(MAX_THREADS, 1)
 bgemm_tc_kernel(TcParams p)
 {
@@ -485,8 +571,12 @@ bgemm_tc_kernel(TcParams p)
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
 
-    const int CH = p.wpr >> 2;                                      // 128-bit chunks along K = pipeline steps
+    const int CH = p.wpr >> 2;                                      // 128-bit chunks along K
+    constexpr bool fp4 = FP4;                                       // 4-bit operand form (p.fp4)
+    const int STEPS = p.steps;                                      // pipeline steps: chunks, or pairs of chunks (4-bit form)
+    const int step_words = fp4 ? 2 * STAGE_WORDS : STAGE_WORDS;     // packed words of K per pipeline step
     const int split_word = (p.nseg == 2) ? (a.I >> 5) : p.wpr;      // first word of the second column segment
+    if (fp4 && warp < 4) write_unit_scales(tmem_base, p.sf_col, warp);      // (expander warps; ordered before the MMAs by their arrivals)
 
     if (warp < mma_warp) {
         // ---- expanders: G groups of EXP threads take the steps in turn; inside a group thread r owns operand
@@ -532,8 +622,15 @@ bgemm_tc_kernel(TcParams p)
         const uint4 zero = make_uint4(0, 0, 0, 0);
         const bool weight_row = r_all < MT * TILE_M;
         if (!weight_row) grid_dependency_wait();
-        uint4 cur = (src && grp < CH) ? load_row_chunk(src + grp, weight_row) : zero;       // own steps: grp, grp + G, ..
-        uint4 nxt = (src && grp + G < CH) ? load_row_chunk(src + grp + G, weight_row) : zero;
+        // chunk(s) of pipeline step c: c, or 2 c and 2 c + 1 in the 4-bit form (a chunk past the end of the row is zeros)
+        auto load_step = [&](int c, uint4& lo, uint4& hi) {
+            const int c0 = fp4 ? 2 * c : c;
+            lo = (src && c < STEPS && c0 < CH) ? load_row_chunk(src + c0, weight_row) : zero;
+            hi = (fp4 && src && c < STEPS && c0 + 1 < CH) ? load_row_chunk(src + c0 + 1, weight_row) : zero;
+        };
+        uint4 cur, cur2, nxt, nxt2;
+        load_step(grp, cur, cur2);                                  // own steps: grp, grp + G, ..
+        load_step(grp + G, nxt, nxt2);
         if (weight_row) grid_dependency_wait();
         const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
         uint32_t off[8];                                            // swizzled position of chunk j: j xor (row mod 8)
@@ -555,20 +652,25 @@ bgemm_tc_kernel(TcParams p)
         bool coef_pending = coef_dst != nullptr;
         int buf = grp;                                              // G <= S
         uint32_t empty_parity = 1;                                  // parity that means "never used" on the first lap
-        for (int c = grp; c < CH; c += G) {
-            const uint4 v = cur;
-            cur = nxt;
-            nxt = (src && c + 2 * G < CH) ? load_row_chunk(src + c + 2 * G, weight_row) : zero;
+        for (int c = grp; c < STEPS; c += G) {
+            const uint4 v = cur, v2 = cur2;
+            cur = nxt; cur2 = nxt2;
+            load_step(c + 2 * G, nxt, nxt2);
             // the MMAs that read this buffer one lap ago must have completed
             if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; break; }
             if (writes) {
-                expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, v, mul, m_sign, m_half);
+                if (fp4) {
+                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off, v);
+                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off + 4, v2);
+                } else {
+                    expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, v, mul, m_sign, m_half);
+                }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
             if (coef_pending) {
                 *coef_dst = coef_val;
-                if (has_corr) sBcorr[(r_all - MT * TILE_M) / KA] = -(float)(p.wpr * 32 - a.n) * corr_sum;
+                if (has_corr) sBcorr[(r_all - MT * TILE_M) / KA] = -(float)p.pad * corr_sum;
                 coef_pending = false;
             }
             buf += G;
@@ -576,30 +678,42 @@ bgemm_tc_kernel(TcParams p)
         }
         if (coef_pending) {                                         // (a group without a step of its own)
             *coef_dst = coef_val;
-            if (has_corr) sBcorr[(r_all - MT * TILE_M) / KA] = -(float)(p.wpr * 32 - a.n) * corr_sum;
+            if (has_corr) sBcorr[(r_all - MT * TILE_M) / KA] = -(float)p.pad * corr_sum;
         }
     } else if (lane == 0) {
         // ---- MMA issuer ----
-        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+        // instruction descriptor: int8 (s32 accumulators, signed 8-bit operands), or block-scaled E2M1 (operand format 1,
+        // scale format E8M0); N >> 3 at bit 17, M >> 4 at bit 24, both operands K-major
+        const uint32_t idesc = fp4 ? ((1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | (1u << 23) | ((uint32_t)(TILE_M >> 4) << 24))
+                                   : ((2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24));
         const uint64_t desc_base = smem_desc(smem_u32(stage_base)); // descriptor of stage 0, tile 0, word 0
+        const uint32_t sf_tmem = tmem_base + (uint32_t)p.sf_col;
         int buf = 0;
         uint32_t full_parity = 0;
-        for (int c = 0; c < CH; ++c) {
+        for (int c = 0; c < STEPS; ++c) {
             if (!mbar_wait(smem_u32(&full_bar[buf]), full_parity)) { *failed = 1; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             // descriptors of the stage: start addresses are below 256 KiB, so adding to the low word never carries
             const uint64_t adesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
             const uint64_t bdesc0 = adesc0 + (uint64_t)(a_stage_bytes >> 4);
-            const int word0 = c * STAGE_WORDS;
-            if (word0 >= split_word || word0 + STAGE_WORDS <= split_word) {
-                // the whole stage lies in one column segment (always, unless a GRU's input width is not a multiple of 128)
+            const int word0 = c * step_words;
+            if (fp4 || word0 >= split_word || word0 + step_words <= split_word) {
+                // the whole stage lies in one column segment (always in the 4-bit form; else unless a GRU's input width is
+                // not a multiple of 128)
                 const int seg = word0 >= split_word ? 1 : 0;
                 const uint32_t acc_first = (word0 != 0 && word0 != split_word) ? 1u : 0u;
                 const uint32_t hi = (uint32_t)(desc_base >> 32);
-                mma_i8_stage(tmem_base + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first);
-                if (MT == 2)
-                    mma_i8_stage(tmem_base + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi, idesc,
-                                 acc_first);
+                if (fp4) {
+                    mma_mxf4_stage(tmem_base + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first, sf_tmem);
+                    if (MT == 2)
+                        mma_mxf4_stage(tmem_base + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi,
+                                       idesc, acc_first, sf_tmem);
+                } else {
+                    mma_i8_stage(tmem_base + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first);
+                    if (MT == 2)
+                        mma_i8_stage(tmem_base + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi,
+                                     idesc, acc_first);
+                }
             } else {
 #pragma unroll
                 for (int qq = 0; qq < STAGE_WORDS; ++qq) {
@@ -653,7 +767,7 @@ bgemm_tc_kernel(TcParams p)
 // expansion and the MMAs of the next one (bound by shared-memory traffic).  The stage pipeline runs on across
 // tiles; "accumulator full" barriers are signalled by tcgen05.commit after the last MMA of a tile,
 // "accumulator empty" ones by the epilogue warps after their last read of tensor memory.
-template <int KA>
+template <int KA, bool FP4>
 __global__ void __launch_bounds__(MAX_THREADS, 1)
 bgemm_tc_persistent_kernel(TcParams p)
 {
@@ -668,7 +782,10 @@ bgemm_tc_persistent_kernel(TcParams p)
     const int a_stage_bytes = MT * TILE_M * 128;
     const int stage_bytes = a_stage_bytes + n_mma * 128;
     const int acc_cols = MT * p.nseg * n_mma;       // columns of one accumulator buffer
-    const int CH = p.wpr >> 2;                      // pipeline steps per tile
+    const int CH = p.wpr >> 2;                      // 128-bit chunks along K
+    constexpr bool fp4 = FP4;                       // 4-bit operand form (p.fp4)
+    const int STEPS = p.steps;                      // pipeline steps per tile: chunks, or pairs of chunks (4-bit form)
+    const int step_words = fp4 ? 2 * STAGE_WORDS : STAGE_WORDS;
     const int split_word = (p.nseg == 2) ? (a.I >> 5) : p.wpr;
     const int ntiles = p.ntiles, MG = p.mgroups, tile_step = (int)gridDim.x;
 
@@ -705,6 +822,7 @@ bgemm_tc_persistent_kernel(TcParams p)
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+    if (fp4 && warp < 4) write_unit_scales(tmem_base, p.sf_col, warp);      // (expander warps; ordered before the MMAs by their arrivals)
 
     if (warp < mma_warp) {
         // ---- expanders: thread r of a group owns operand row r of every tile; the groups take the steps of the
@@ -751,25 +869,36 @@ bgemm_tc_persistent_kernel(TcParams p)
         // load cursor: runs two of the group's steps ahead of the expansion, across tile boundaries
         int pf_tile = (int)blockIdx.x, pf_c = grp;
         const uint4* pf_src = row_of(pf_tile);
-        auto pf_load = [&]() -> uint4 {
-            while (pf_c >= CH) { pf_c -= CH; pf_tile += tile_step; pf_src = row_of(pf_tile); }
-            const uint4 v = pf_src ? load_row_chunk(pf_src + pf_c, is_a) : zero;
+        // chunk(s) of the cursor's step: one, or a pair in the 4-bit form (a chunk past the end of the row is zeros)
+        auto pf_load = [&](uint4& lo, uint4& hi) {
+            while (pf_c >= STEPS) { pf_c -= STEPS; pf_tile += tile_step; pf_src = row_of(pf_tile); }
+            const int c0 = fp4 ? 2 * pf_c : pf_c;
+            lo = pf_src ? load_row_chunk(pf_src + c0, is_a) : zero;
+            hi = (fp4 && pf_src && c0 + 1 < CH) ? load_row_chunk(pf_src + c0 + 1, is_a) : zero;
             pf_c += G;
-            return v;
         };
         const int my_tiles = (ntiles - (int)blockIdx.x + tile_step - 1) / tile_step;
-        const int total = my_tiles * CH;
+        const int total = my_tiles * STEPS;
         if (!is_a) grid_dependency_wait();                          // activation planes come from the preceding kernel
-        uint4 cur = pf_load(), nxt = pf_load();
+        uint4 cur, cur2, nxt, nxt2;
+        pf_load(cur, cur2);
+        pf_load(nxt, nxt2);
         if (is_a) grid_dependency_wait();
         int buf = grp;                                              // G <= S
         uint32_t empty_parity = 1;
         for (int q = grp; q < total; q += G) {
-            const uint4 v = cur;
-            cur = nxt;
-            nxt = pf_load();
+            const uint4 v = cur, v2 = cur2;
+            cur = nxt; cur2 = nxt2;
+            pf_load(nxt, nxt2);
             if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity, failed)) { *failed = 1; break; }
-            if (writes) expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, v, mul, m_sign, m_half);
+            if (writes) {
+                if (fp4) {
+                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off, v);
+                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off + 4, v2);
+                } else {
+                    expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, v, mul, m_sign, m_half);
+                }
+            }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
             buf += G;
@@ -778,8 +907,10 @@ bgemm_tc_persistent_kernel(TcParams p)
     } else if (warp == mma_warp) {
         if (lane == 0) {
             // ---- MMA issuer ----
-            const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+            const uint32_t idesc = fp4 ? ((1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | (1u << 23) | ((uint32_t)(TILE_M >> 4) << 24))
+                                       : ((2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24));
             const uint64_t desc_base = smem_desc(smem_u32(stage_base));
+            const uint32_t sf_tmem = tmem_base + (uint32_t)p.sf_col;
             int buf = 0;
             uint32_t full_parity = 0;
             bool ok = true;
@@ -791,20 +922,27 @@ bgemm_tc_persistent_kernel(TcParams p)
                 if (!mbar_wait(smem_u32(&tempty_bar[ab]), (use & 1u) ^ 1u)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t acc = tmem_base + (uint32_t)(ab * acc_cols);
-                for (int c = 0; c < CH; ++c) {
+                for (int c = 0; c < STEPS; ++c) {
                     if (!mbar_wait(smem_u32(&full_bar[buf]), full_parity)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t adesc0 = desc_base + (uint64_t)((buf * stage_bytes) >> 4);
                     const uint64_t bdesc0 = adesc0 + (uint64_t)(a_stage_bytes >> 4);
-                    const int word0 = c * STAGE_WORDS;
-                    if (word0 >= split_word || word0 + STAGE_WORDS <= split_word) {
+                    const int word0 = c * step_words;
+                    if (fp4 || word0 >= split_word || word0 + step_words <= split_word) {
                         const int seg = word0 >= split_word ? 1 : 0;
                         const uint32_t acc_first = (word0 != 0 && word0 != split_word) ? 1u : 0u;
                         const uint32_t hi = (uint32_t)(desc_base >> 32);
-                        mma_i8_stage(acc + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first);
-                        if (MT == 2)
-                            mma_i8_stage(acc + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi, idesc,
-                                         acc_first);
+                        if (fp4) {
+                            mma_mxf4_stage(acc + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first, sf_tmem);
+                            if (MT == 2)
+                                mma_mxf4_stage(acc + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi,
+                                               idesc, acc_first, sf_tmem);
+                        } else {
+                            mma_i8_stage(acc + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first);
+                            if (MT == 2)
+                                mma_i8_stage(acc + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi, idesc,
+                                             acc_first);
+                        }
                     } else {
 #pragma unroll
                         for (int qq = 0; qq < STAGE_WORDS; ++qq) {
@@ -850,7 +988,7 @@ bgemm_tc_persistent_kernel(TcParams p)
                     if (j == 0) {
                         float sum = 0.0f;
                         for (int jj = 0; jj < KA; ++jj) sum += use_b ? __ldcg(a.xbeta + (size_t)b * KA + jj) : 0.0f;
-                        sBcorr[e] = -(float)(p.wpr * 32 - a.n) * sum;
+                        sBcorr[e] = -(float)p.pad * sum;
                     }
                 }
             }
@@ -921,8 +1059,15 @@ bool plan_persistent(const TcParams& base, int mtiles, int btiles, TcPlan* out)
     // GRU's two column segments at N = 192) the MMAs of the next tile wait for the epilogue, but its stages are expanded
     // meanwhile and the CTA pays its set-up once: still ahead of three waves of the plain form (measured)
     p.nbuf = (2 * acc_cols > 512) ? 1 : 2;
+    // 4-bit operands where the scale factors' 16 tensor-memory columns fit beside the accumulator buffers and a GRU's
+    // column split falls on a pipeline step (256 bit positions)
+    const int CH = p.wpr >> 2;
+    p.fp4 = (p.nbuf * acc_cols + 16 <= 512 && (p.nseg == 1 || p.a.I % 256 == 0)) ? 1 : 0;
+    p.sf_col = p.nbuf * acc_cols;
+    p.steps = p.fp4 ? (CH + 1) / 2 : CH;
+    p.pad = p.wpr * 32 - p.a.n + ((p.fp4 && (CH & 1)) ? 128 : 0);
     int cols = 32;
-    while (cols < p.nbuf * acc_cols) cols <<= 1;
+    while (cols < p.nbuf * acc_cols + (p.fp4 ? 16 : 0)) cols <<= 1;
     p.tmem_cols = cols;
     const size_t stage = (size_t)128 * (TILE_M + p.n_mma);
     p.yt_bytes = (int)(((size_t)p.nseg * TILE_M * (p.TB + 1) * 4 + 15) / 16 * 16);
@@ -973,8 +1118,16 @@ bool plan(const GemmArgs& a, TcPlan* out)
     // with one M tile per CTA and more tiles than SMs, the persistent form hides the epilogues; with two M tiles
     // per CTA the plain form's lower shared-memory traffic per MMA counts for more (measured)
     if (p.MT == 1 && plan_persistent(p, mtiles, btiles, out)) return true;
+    // 4-bit operands where the scale factors' 16 tensor-memory columns fit beside the accumulators and a GRU's column
+    // split falls on a pipeline step (256 bit positions)
+    const int acc_cols = p.MT * p.nseg * p.n_mma;
+    const int CH = p.wpr >> 2;
+    p.fp4 = (acc_cols + 16 <= 512 && (p.nseg == 1 || a.I % 256 == 0)) ? 1 : 0;
+    p.sf_col = acc_cols;
+    p.steps = p.fp4 ? (CH + 1) / 2 : CH;
+    p.pad = p.wpr * 32 - a.n + ((p.fp4 && (CH & 1)) ? 128 : 0);
     int cols = 32;
-    while (cols < p.MT * p.nseg * p.n_mma) cols <<= 1;
+    while (cols < acc_cols + (p.fp4 ? 16 : 0)) cols <<= 1;
     if (cols > 512) return false;
     p.tmem_cols = cols;
     const size_t stage = (size_t)128 * (p.MT * TILE_M + p.n_mma);
@@ -997,7 +1150,8 @@ bool plan(const GemmArgs& a, TcPlan* out)
 template <int KA>
 amq_status launch_ka(const TcPlan& pl, cudaStream_t st)
 {
-    auto kernel = pl.persistent ? bgemm_tc_persistent_kernel<KA> : bgemm_tc_kernel<KA>;
+    auto kernel = pl.persistent ? (pl.p.fp4 ? bgemm_tc_persistent_kernel<KA, true> : bgemm_tc_persistent_kernel<KA, false>)
+                                : (pl.p.fp4 ? bgemm_tc_kernel<KA, true> : bgemm_tc_kernel<KA, false>);
     AMQ_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
     if (pl.p.a.overlap_with_previous) {
         cudaLaunchConfig_t cfg{};

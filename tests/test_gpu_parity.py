@@ -228,6 +228,8 @@ CELL_CASES = [
     ("lstm", 40, 640, 4, 4, 70),          # 160 tiles: gate epilogues of the persistent tensor-core kernel
     ("gru", 64, 800, 4, 1, 200),
     ("gru", 32, 1500, 4, 4, 40),          # 150 tiles, two column segments of N = 192: persistent kernel, one accumulator buffer
+    ("gru", 256, 200, 2, 3, 24),          # column split on a pipeline step of the 4-bit operand form (256 bit positions)
+    ("gru", 256, 1600, 4, 3, 40),         # the same in the persistent kernel, odd number of 128-bit chunks per row
     # batch 1 goes through the persistent weight-stationary kernel
     ("lstm", 1024, 1024, 2, 2, 1),        # the hidden-1024 layer of the benchmark, one step
     ("lstm", 1536, 1024, 3, 3, 1),        # n = 2560: sixteen elements per thread
