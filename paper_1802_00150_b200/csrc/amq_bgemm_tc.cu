@@ -552,42 +552,32 @@ bgemm_tc_kernel(TcParams p)
     float* sBeta = sAlpha + 2 * TILE_M;                             // [TB][KA]  coefficients of the activation tile
     float* sBcorr = sBeta + 256;                                    // [TB]      -pad * their sum per batch entry
 
-    if (tid == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(smem_u32(&full_bar[s]), (uint32_t)EXP);
-            mbar_init(smem_u32(&empty_bar[s]), 1);
-        }
-        mbar_init(smem_u32(done_bar), 1);
-        *failed = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == mma_warp) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem_base = *tmem_slot;
-
     const int CH = p.wpr >> 2;                                      // 128-bit chunks along K
     constexpr bool fp4 = FP4;                                       // 4-bit operand form (p.fp4)
     const int STEPS = p.steps;                                      // pipeline steps: chunks, or pairs of chunks (4-bit form)
     const int step_words = fp4 ? 2 * STAGE_WORDS : STAGE_WORDS;     // packed words of K per pipeline step
     const int split_word = (p.nseg == 2) ? (a.I >> 5) : p.wpr;      // first word of the second column segment
-    if (fp4 && warp < 4) write_unit_scales(tmem_base, p.sf_col, warp);      // (expander warps; ordered before the MMAs by their arrivals)
-
-    if (warp < mma_warp) {
-        // ---- expanders: G groups of EXP threads take the steps in turn; inside a group thread r owns operand
-        //      row r (A plane-rows first, then the B rows) ----
-        const int grp = (tid >= EXP ? 1 : 0) + (tid >= 2 * EXP ? 1 : 0) + (tid >= 3 * EXP ? 1 : 0), r_all = tid - grp * EXP;   // G <= 4
-        const uint4* src = nullptr;
-        uint32_t dst0;                                              // shared address of the row in stage 0
-        const float* coef_src = nullptr;                            // the row's coefficient, staged for the epilogue
-        float* coef_dst = nullptr;
-        const float* corr_src = nullptr;                            // first of the KA coefficients of a batch entry
-        if (r_all < MT * TILE_M) {
+    // ---- expanders, before the CTA's set-up barrier: G groups of EXP threads take the steps in turn; inside a group thread r
+    //      owns operand row r (A plane-rows first, then the B rows).  The row bookkeeping and the first loads come first, so
+    //      that their latency runs beside the barrier initialisation and the tensor-memory allocation ----
+    const bool expander = warp < mma_warp;
+    const int grp = (tid >= EXP ? 1 : 0) + (tid >= 2 * EXP ? 1 : 0) + (tid >= 3 * EXP ? 1 : 0), r_all = tid - grp * EXP;   // G <= 4
+    const uint4* src = nullptr;
+    uint32_t dst0 = 0;                                              // shared address of the row in stage 0
+    const float* coef_src = nullptr;                                // the row's coefficient, staged for the epilogue
+    float* coef_dst = nullptr;
+    const float* corr_src = nullptr;                                // first of the KA coefficients of a batch entry
+    const bool weight_row = r_all < MT * TILE_M;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    // chunk(s) of pipeline step c: c, or 2 c and 2 c + 1 in the 4-bit form (a chunk past the end of the row is zeros)
+    auto load_step = [&](int c, uint4& lo, uint4& hi) {
+        const int c0 = fp4 ? 2 * c : c;
+        lo = (src && c < STEPS && c0 < CH) ? load_row_chunk(src + c0, weight_row) : zero;
+        hi = (fp4 && src && c < STEPS && c0 + 1 < CH) ? load_row_chunk(src + c0 + 1, weight_row) : zero;
+    };
+    uint4 cur = zero, cur2 = zero, nxt = zero, nxt2 = zero;
+    if (expander) {
+        if (weight_row) {
             const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
             size_t prow = 0;                                        // plane-row index in Wcodes / Walpha
             if (r < TMp) {
@@ -616,21 +606,35 @@ bgemm_tc_kernel(TcParams p)
                 if (j == 0) corr_src = coef_src;
             }
         }
-        // weight rows are fetched at once, before anything else is set up (their latency is the longest item of a
-        // CTA's start-up); everything the preceding kernel of the stream may have written (the activation planes and
-        // their coefficients, the state) is read after the wait
-        const uint4 zero = make_uint4(0, 0, 0, 0);
-        const bool weight_row = r_all < MT * TILE_M;
+        // weight rows are fetched at once (no kernel of a chain writes them); everything the preceding kernel of the
+        // stream may have written (the activation planes and their coefficients, the state) is read after the wait
         if (!weight_row) grid_dependency_wait();
-        // chunk(s) of pipeline step c: c, or 2 c and 2 c + 1 in the 4-bit form (a chunk past the end of the row is zeros)
-        auto load_step = [&](int c, uint4& lo, uint4& hi) {
-            const int c0 = fp4 ? 2 * c : c;
-            lo = (src && c < STEPS && c0 < CH) ? load_row_chunk(src + c0, weight_row) : zero;
-            hi = (fp4 && src && c < STEPS && c0 + 1 < CH) ? load_row_chunk(src + c0 + 1, weight_row) : zero;
-        };
-        uint4 cur, cur2, nxt, nxt2;
         load_step(grp, cur, cur2);                                  // own steps: grp, grp + G, ..
         load_step(grp + G, nxt, nxt2);
+    }
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), (uint32_t)EXP);
+            mbar_init(smem_u32(&empty_bar[s]), 1);
+        }
+        mbar_init(smem_u32(done_bar), 1);
+        *failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == mma_warp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(smem_u32(tmem_slot)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (fp4 && warp < 4) write_unit_scales(tmem_base, p.sf_col, warp);      // (expander warps; ordered before the MMAs by their arrivals)
+
+    if (expander) {
         if (weight_row) grid_dependency_wait();
         const bool writes = r_all < MT * TILE_M + n_mma;            // threads past the last row only arrive
         uint32_t off[8];                                            // swizzled position of chunk j: j xor (row mod 8)
