@@ -252,6 +252,20 @@ __device__ __forceinline__ uint4 load_row_chunk(const uint4* p, bool weight_row)
     return weight_row ? __ldg(p) : __ldcg(p);       // weights are constant; activation planes: see above
 }
 
+// Two consecutive chunks of a packed row (32 bytes, 32-byte aligned) in one 256-bit load.  A warp-wide load of 16 bytes from
+// 32 different rows costs the load/store unit about as much as one of 32 bytes (measured: the shared-memory stores of the
+// expansion, which queue behind the loads, ran at 34 bytes per clock per SM beside two 16-byte loads per row and step, at
+// 53-67 beside one 32-byte load), so the 4-bit form, whose pipeline step consumes 32 bytes per row, loads them at once.
+__device__ __forceinline__ void load_row_chunk_pair(const uint4* p, bool weight_row, uint4& lo, uint4& hi)
+{
+    if (weight_row)
+        asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w), "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w) : "l"(p));
+    else
+        asm volatile("ld.global.cg.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w), "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w) : "l"(p) : "memory");
+}
+
 // one 128-bit chunk of a packed row -> its 128 operand bytes (eight 16-byte pieces at the swizzled offsets `off`)
 __device__ __forceinline__ void expand_chunk(uint32_t base, const uint32_t (&off)[8], const uint4& v, const uint32_t (&mul)[7],
                                              uint32_t m_sign, uint32_t m_half)
@@ -572,6 +586,10 @@ bgemm_tc_kernel(TcParams p)
     // chunk(s) of pipeline step c: c, or 2 c and 2 c + 1 in the 4-bit form (a chunk past the end of the row is zeros)
     auto load_step = [&](int c, uint4& lo, uint4& hi) {
         const int c0 = fp4 ? 2 * c : c;
+        if (fp4 && src && c0 + 1 < CH && (reinterpret_cast<uintptr_t>(src) & 31) == 0) {      // (c0 + 1 < CH implies c < STEPS)
+            load_row_chunk_pair(src + c0, weight_row, lo, hi);
+            return;
+        }
         lo = (src && c < STEPS && c0 < CH) ? load_row_chunk(src + c0, weight_row) : zero;
         hi = (fp4 && src && c < STEPS && c0 + 1 < CH) ? load_row_chunk(src + c0 + 1, weight_row) : zero;
     };
@@ -877,8 +895,12 @@ bgemm_tc_persistent_kernel(TcParams p)
         auto pf_load = [&](uint4& lo, uint4& hi) {
             while (pf_c >= STEPS) { pf_c -= STEPS; pf_tile += tile_step; pf_src = row_of(pf_tile); }
             const int c0 = fp4 ? 2 * pf_c : pf_c;
-            lo = pf_src ? load_row_chunk(pf_src + c0, is_a) : zero;
-            hi = (fp4 && pf_src && c0 + 1 < CH) ? load_row_chunk(pf_src + c0 + 1, is_a) : zero;
+            if (fp4 && pf_src && c0 + 1 < CH && (reinterpret_cast<uintptr_t>(pf_src) & 31) == 0) {
+                load_row_chunk_pair(pf_src + c0, is_a, lo, hi);
+            } else {
+                lo = pf_src ? load_row_chunk(pf_src + c0, is_a) : zero;
+                hi = (fp4 && pf_src && c0 + 1 < CH) ? load_row_chunk(pf_src + c0 + 1, is_a) : zero;
+            }
             pf_c += G;
         };
         const int my_tiles = (ntiles - (int)blockIdx.x + tile_step - 1) / tile_step;
