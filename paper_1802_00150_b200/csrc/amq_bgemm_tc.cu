@@ -583,15 +583,17 @@ bgemm_tc_kernel(TcParams p)
     const float* corr_src = nullptr;                                // first of the KA coefficients of a batch entry
     const bool weight_row = r_all < MT * TILE_M;
     const uint4 zero = make_uint4(0, 0, 0, 0);
-    // chunk(s) of pipeline step c: c, or 2 c and 2 c + 1 in the 4-bit form (a chunk past the end of the row is zeros)
-    auto load_step = [&](int c, uint4& lo, uint4& hi) {
-        const int c0 = fp4 ? 2 * c : c;
-        if (fp4 && src && c0 + 1 < CH && (reinterpret_cast<uintptr_t>(src) & 31) == 0) {      // (c0 + 1 < CH implies c < STEPS)
+    // A group's unit of work is a pair of 128-bit chunks of its rows (chunks 2 q and 2 q + 1; one past the end of the row is
+    // zeros): one pipeline step in the 4-bit form, two consecutive ones otherwise.  Where the row is 32-byte aligned the
+    // pair comes in one load.
+    auto load_pair = [&](int q, uint4& lo, uint4& hi) {
+        const int c0 = 2 * q;
+        if (src && c0 + 1 < CH && (reinterpret_cast<uintptr_t>(src) & 31) == 0) {
             load_row_chunk_pair(src + c0, weight_row, lo, hi);
             return;
         }
-        lo = (src && c < STEPS && c0 < CH) ? load_row_chunk(src + c0, weight_row) : zero;
-        hi = (fp4 && src && c < STEPS && c0 + 1 < CH) ? load_row_chunk(src + c0 + 1, weight_row) : zero;
+        lo = (src && c0 < CH) ? load_row_chunk(src + c0, weight_row) : zero;
+        hi = (src && c0 + 1 < CH) ? load_row_chunk(src + c0 + 1, weight_row) : zero;
     };
     uint4 cur = zero, cur2 = zero, nxt = zero, nxt2 = zero;
     if (expander) {
@@ -627,8 +629,8 @@ bgemm_tc_kernel(TcParams p)
         // weight rows are fetched at once (no kernel of a chain writes them); everything the preceding kernel of the
         // stream may have written (the activation planes and their coefficients, the state) is read after the wait
         if (!weight_row) grid_dependency_wait();
-        load_step(grp, cur, cur2);                                  // own steps: grp, grp + G, ..
-        load_step(grp + G, nxt, nxt2);
+        load_pair(grp, cur, cur2);                                  // own pairs: grp, grp + G, ..
+        load_pair(grp + G, nxt, nxt2);
     }
 
     if (tid == 0) {
@@ -672,31 +674,47 @@ bgemm_tc_kernel(TcParams p)
             for (int jj = 0; jj < KA; ++jj) corr_sum += __ldcg(corr_src + jj);
         }
         bool coef_pending = coef_dst != nullptr;
-        int buf = grp;                                              // G <= S
+        const int PAIRS = (CH + 1) >> 1;
+        int buf = fp4 ? grp : 2 * grp;                              // stage buffer of the pair's first pipeline step
         uint32_t empty_parity = 1;                                  // parity that means "never used" on the first lap
-        for (int c = grp; c < STEPS; c += G) {
-            const uint4 v = cur, v2 = cur2;
-            cur = nxt; cur2 = nxt2;
-            load_step(c + 2 * G, nxt, nxt2);
-            // the MMAs that read this buffer one lap ago must have completed
-            if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; break; }
+        auto advance = [&](int d) {
+            buf += d;
+            while (buf >= S) { buf -= S; empty_parity ^= 1u; }
+        };
+        advance(0);
+        bool go_on = true;
+        // one pipeline step: the MMAs that read this buffer one lap ago must have completed; expand; hand over
+        auto step = [&](const uint4& lo, const uint4& hi) {
+            if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; go_on = false; return; }
             if (writes) {
                 if (fp4) {
-                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off, v);
-                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off + 4, v2);
+                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off, lo);
+                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off + 4, hi);
                 } else {
-                    expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, v, mul, m_sign, m_half);
+                    expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, lo, mul, m_sign, m_half);
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
+        };
+        for (int q = grp; q < PAIRS && go_on; q += G) {
+            const uint4 v = cur, v2 = cur2;
+            cur = nxt; cur2 = nxt2;
+            load_pair(q + 2 * G, nxt, nxt2);
+            step(v, v2);
+            if (!go_on) break;
             if (coef_pending) {
                 *coef_dst = coef_val;
                 if (has_corr) sBcorr[(r_all - MT * TILE_M) / KA] = -(float)p.pad * corr_sum;
                 coef_pending = false;
             }
-            buf += G;
-            if (buf >= S) { buf -= S; empty_parity ^= 1u; }
+            if (fp4) {
+                advance(G);
+            } else {
+                advance(1);
+                if (2 * q + 1 < CH) step(v2, v2);
+                advance(2 * G - 1);
+            }
         }
         if (coef_pending) {                                         // (a group without a step of its own)
             *coef_dst = coef_val;
