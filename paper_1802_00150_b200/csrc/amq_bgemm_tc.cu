@@ -1121,9 +1121,11 @@ bool plan_persistent(const TcParams& base, int mtiles, int btiles, TcPlan* out)
     if (S < 2) return false;
     p.nstages = S;
     p.expanders = (TILE_M + p.n_mma + 31) / 32 * 32;
-    // one expander group and eight epilogue warps
+    // one expander group; eight epilogue warps, or up to sixteen where the MMAs of the next tile have to wait for the
+    // epilogue (one accumulator buffer; measured: C4 timestep 53.7 -> 50.3 us, nothing gained with two buffers)
     p.groups = 1;
-    p.epi_warps = 8;
+    p.epi_warps = (p.nbuf == 1) ? 16 : 8;
+    while (p.epi_warps > 4 && p.groups * p.expanders + 32 + 32 * p.epi_warps > MAX_THREADS) p.epi_warps -= 4;
     if (p.groups * p.expanders + 32 + 32 * p.epi_warps > MAX_THREADS) return false;
     out->p = p;
     out->smem = S * stage + fixed;
@@ -1160,8 +1162,11 @@ bool plan(const GemmArgs& a, TcPlan* out)
     p.mask_half = 0x40404040u;
     p.MT = (2 * p.nseg * p.n_mma <= 512 && (long long)(mtiles / 2) * btiles >= 2 * sm_count()) ? 2 : 1;
     // with one M tile per CTA and more tiles than SMs, the persistent form hides the epilogues; with two M tiles
-    // per CTA the plain form's lower shared-memory traffic per MMA counts for more (measured)
-    if (p.MT == 1 && plan_persistent(p, mtiles, btiles, out)) return true;
+    // per CTA the plain form's lower shared-memory traffic per MMA counts for more (measured), unless their accumulators
+    // leave no room for the scale factors of the 4-bit form and one M tile per CTA does (C5: 142 us plain with int8
+    // operands, 123 us persistent with 4-bit ones)
+    const bool two_tiles_4bit = 2 * p.nseg * p.n_mma + 16 <= 512 && (p.nseg == 1 || a.I % 256 == 0);
+    if ((p.MT == 1 || !two_tiles_4bit) && plan_persistent(p, mtiles, btiles, out) && (p.MT == 1 || out->p.fp4)) return true;
     // 4-bit operands where the scale factors' 16 tensor-memory columns fit beside the accumulators and a GRU's column
     // split falls on a pipeline step (256 bit positions)
     const int acc_cols = p.MT * p.nseg * p.n_mma;

@@ -159,6 +159,8 @@ GEMM_CASES = [
     (2500, 300, 4, 4, 70),               # more tiles than SMs, one M tile per CTA: the persistent tensor-core kernel
     (2500, 100, 4, 4, 70),               # the same with a single pipeline step per tile
     (6144, 200, 2, 3, 250),              # 384 tiles, ragged last batch tile
+    (25000, 200, 3, 2, 128),             # N = 256: two M tiles per CTA would fill tensor memory; persistent kernel, 4-bit operands,
+                                         # one accumulator buffer, sixteen epilogue warps
     # batch 1: the streaming matrix-vector kernel (segments of 1..32 lanes per row, one or two chunks per lane)
     (300, 8192, 3, 3, 1),
     (1000, 1024, 2, 3, 1),
