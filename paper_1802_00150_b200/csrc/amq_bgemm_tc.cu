@@ -1010,32 +1010,58 @@ bgemm_tc_persistent_kernel(TcParams p)
         const int tid_e = tid - epi_warp0 * 32, nth_e = EW * 32;
         const int quarter = warp & 3, slot = (warp - epi_warp0) >> 2, nslots = EW >> 2;
         grid_dependency_wait();                                     // coefficients and state come from preceding kernels
+        // Coefficients of a tile, staged in shared memory for the first half of the epilogue: alpha per plane-row, beta
+        // per (entry, plane), -pad * sum_j beta_j per entry.  The global loads for the next tile are issued before the
+        // second half of the epilogue of this one and their values stored after it, so that their latency is off the
+        // tile-to-tile chain of the epilogue warps (at most one plane-row and two activation columns per thread:
+        // one M tile per CTA, N <= 256, at least 128 epilogue threads).
+        float c_alpha = 0.0f, c_beta[2] = {0.0f, 0.0f}, c_corr[2] = {0.0f, 0.0f};
+        auto coef_load = [&](int tile) {
+            const int bt = tile / MG, mg = tile - bt * MG;
+            const int u0 = mg * p.UT * MT, b0 = bt * p.TB;
+            c_alpha = 0.0f;
+            if (tid_e < MT * TILE_M) {
+                const int mt = tid_e >> 7, r = tid_e & (TILE_M - 1);
+                const int l = div_small(r, k_w), i = r - l * k_w;
+                const int lg = div_small(l, p.gates);
+                const int u = u0 + mt * p.UT + lg, gate = l - lg * p.gates;
+                if (r < TMp && u < p.units) c_alpha = __ldg(a.Walpha + ((size_t)gate * p.units + u) * k_w + i);
+            }
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int idx = tid_e + k * nth_e;
+                c_beta[k] = 0.0f; c_corr[k] = 0.0f;
+                if (idx < n_mma) {
+                    const int e = idx / KA, j = idx - e * KA, b = b0 + e;
+                    if (b < a.batch) {
+                        c_beta[k] = __ldcg(a.xbeta + (size_t)b * KA + j);
+                        if (j == 0) {
+                            float sum = 0.0f;
+                            for (int jj = 0; jj < KA; ++jj) sum += __ldcg(a.xbeta + (size_t)b * KA + jj);
+                            c_corr[k] = -(float)p.pad * sum;
+                        }
+                    }
+                }
+            }
+        };
+        auto coef_store = [&]() {
+            if (tid_e < MT * TILE_M) sAlpha[tid_e] = c_alpha;
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int idx = tid_e + k * nth_e;
+                if (idx < n_mma) {
+                    sBeta[idx] = c_beta[k];
+                    if (idx % KA == 0) sBcorr[idx / KA] = c_corr[k];
+                }
+            }
+        };
+        if (a.epilogue != EPI_DOTS && (int)blockIdx.x < ntiles) { coef_load((int)blockIdx.x); coef_store(); }
         int it = 0;
         for (int tile = (int)blockIdx.x; tile < ntiles; tile += tile_step, ++it) {
             const int ab = (p.nbuf == 2) ? (it & 1) : 0;
             const uint32_t use = (p.nbuf == 2) ? (uint32_t)(it >> 1) : (uint32_t)it;
             const int bt = tile / MG, mg = tile - bt * MG;
             const int u0 = mg * p.UT * MT, b0 = bt * p.TB;
-            // coefficients of the tile (every thread is past the previous tile's first half, which read the old ones)
-            if (a.epilogue != EPI_DOTS) {
-                for (int idx = tid_e; idx < MT * TILE_M; idx += nth_e) {
-                    const int mt = idx >> 7, r = idx & (TILE_M - 1);
-                    const int l = div_small(r, k_w), i = r - l * k_w;
-                    const int lg = div_small(l, p.gates);
-                    const int u = u0 + mt * p.UT + lg, gate = l - lg * p.gates;
-                    sAlpha[idx] = (r < TMp && u < p.units) ? __ldg(a.Walpha + ((size_t)gate * p.units + u) * k_w + i) : 0.0f;
-                }
-                for (int idx = tid_e; idx < n_mma; idx += nth_e) {
-                    const int e = idx / KA, j = idx - e * KA, b = b0 + e;
-                    const bool use_b = b < a.batch;
-                    sBeta[idx] = use_b ? __ldcg(a.xbeta + (size_t)b * KA + j) : 0.0f;
-                    if (j == 0) {
-                        float sum = 0.0f;
-                        for (int jj = 0; jj < KA; ++jj) sum += use_b ? __ldcg(a.xbeta + (size_t)b * KA + jj) : 0.0f;
-                        sBcorr[e] = -(float)p.pad * sum;
-                    }
-                }
-            }
             const bool ok = mbar_wait_relaxed(smem_u32(&tfull_bar[ab]), use & 1u, failed);
             __syncwarp();
             // one barrier: the coefficients are visible, every thread has left the previous tile's second half
@@ -1050,8 +1076,11 @@ bgemm_tc_persistent_kernel(TcParams p)
                 asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&tempty_bar[ab])) : "memory");
             if (a.epilogue == EPI_DOTS) continue;
             __syncwarp();
-            epi_bar(nth_e);                                         // the staging array is complete
+            epi_bar(nth_e);                                         // the staging array is complete, the coefficients are read
+            const bool more = tile + tile_step < ntiles;
+            if (more) coef_load(tile + tile_step);
             epilogue_smem_to_global(p, Yt, u0, b0, tid_e, nth_e);
+            if (more) coef_store();                                 // (visible to the others after the next tile's barrier)
             __syncwarp();
         }
     }
