@@ -1,8 +1,11 @@
-// Microbenchmark: how tcgen05.mma (kind::i8, M 128 x N 192 x K 32, both operands in shared memory) and 128-bit
-// shared-memory stores share the shared-memory port.  One thread issues MMAs back to back over a fixed operand tile
-// while `st_threads` other threads stream stores in the access pattern of the operand expansion (own 128-byte row,
-// eight swizzled 16-byte pieces per round) into another region, until the MMAs have completed.  Reported: clocks per
-// MMA and store bytes per clock, each alone and together.  One CTA per SM on every SM; every wait is bounded.
+// Microbenchmark: how tcgen05.mma (kind::i8, M 128 x N 192 x K 32, both operands in shared memory), 128-bit
+// shared-memory stores and the global loads that feed them share the SM's memory pipeline.  One thread issues MMAs back
+// to back over a fixed operand tile while `st_threads` other threads do what the expander threads of the product kernel
+// do, round after round, until the MMAs have completed: (optionally) load 32 bytes of their own packed row from global
+// memory (rows 1 KB apart, L2-resident; as two 16-byte loads or one 256-bit load; 1, 2 or 4 rounds ahead), expand them
+// to 4-bit operands with shifts and masks, store the eight 16-byte pieces of their 128-byte shared-memory row at the
+// swizzled positions, proxy fence.  Reported: clocks per MMA and store bytes per clock, alone and together.  One CTA per
+// SM on every SM; every wait is bounded.
 #include <cstdio>
 #include <cstdlib>
 #include <cstdint>
@@ -26,7 +29,9 @@ constexpr int N_MMA = 192;
 constexpr int OPERAND_BYTES = (128 + 256) * 128;        // A: 128 rows, B: up to 256 rows of 128 bytes
 constexpr int MAX_ROUNDS = 1 << 16;
 
-struct P { int mma_count, st_threads, fence; long long* clk; unsigned long long* rounds; unsigned* err; };
+// mode bits: 1 proxy fence per round, 2 expansion arithmetic, 4 global loads, 16 two rounds ahead, 64 four rounds ahead,
+// 32 one 256-bit load instead of two 128-bit ones
+struct P { const uint4* gsrc; int mma_count, st_threads, fence; long long* clk; unsigned long long* rounds; unsigned* err; };
 
 __global__ void __launch_bounds__(1024, 1) mma_with_stores(P p)
 {
@@ -87,14 +92,67 @@ __global__ void __launch_bounds__(1024, 1) mma_with_stores(P p)
         unsigned off[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) off[j] = (unsigned)((j ^ (r & 7)) << 4);
-        unsigned v = 0x22222222u + r;
         int rounds = 0;
-        while (rounds < MAX_ROUNDS && !mma_done) {
+        const uint4* gsrc = p.gsrc + (size_t)(blockIdx.x * 1024 + r) * 64;
+        auto expand_store = [&](const uint4& a, const uint4& b) {
+            const unsigned w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" :: "r"(base + off[j]), "r"(v + j), "r"(v ^ rounds), "r"(v), "r"(v + rounds) : "memory");
-            if (p.fence) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            ++rounds;
+            for (int j = 0; j < 8; ++j) {
+                const unsigned y0 = ((w[j] << 3) & 0x88888888u) | 0x22222222u;
+                const unsigned y1 = ((w[j] << 2) & 0x88888888u) | 0x22222222u;
+                const unsigned y2 = ((w[j] << 1) & 0x88888888u) | 0x22222222u;
+                const unsigned y3 = (w[j] & 0x88888888u) | 0x22222222u;
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" :: "r"(base + off[j]), "r"(y0), "r"(y1), "r"(y2), "r"(y3) : "memory");
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        };
+        auto load2 = [&](int step, uint4& a, uint4& b) {
+            const uint4* q = gsrc + ((2 * step) & 63);
+            if (p.fence & 32) {
+                asm volatile("ld.global.cg.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                             : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(q) : "memory");
+            } else { a = __ldcg(q); b = __ldcg(q + 1); }
+        };
+        if (p.fence & 16) {
+            // two rounds ahead without register moves: two register sets in turn
+            uint4 a0, b0, a1, b1;
+            load2(0, a0, b0); load2(1, a1, b1);
+            while (rounds < MAX_ROUNDS && !mma_done) {
+                { const uint4 a = a0, b = b0; load2(rounds + 2, a0, b0); expand_store(a, b); }
+                { const uint4 a = a1, b = b1; load2(rounds + 3, a1, b1); expand_store(a, b); }
+                rounds += 2;
+            }
+        } else if (p.fence & 64) {
+            // four rounds ahead
+            uint4 a0, b0, a1, b1, a2, b2, a3, b3;
+            load2(0, a0, b0); load2(1, a1, b1); load2(2, a2, b2); load2(3, a3, b3);
+            while (rounds < MAX_ROUNDS && !mma_done) {
+                { const uint4 a = a0, b = b0; load2(rounds + 4, a0, b0); expand_store(a, b); }
+                { const uint4 a = a1, b = b1; load2(rounds + 5, a1, b1); expand_store(a, b); }
+                { const uint4 a = a2, b = b2; load2(rounds + 6, a2, b2); expand_store(a, b); }
+                { const uint4 a = a3, b = b3; load2(rounds + 7, a3, b3); expand_store(a, b); }
+                rounds += 4;
+            }
+        } else if (!(p.fence & 2)) {
+            // stores of changing register values only
+            const unsigned v = 0x22222222u + r;
+            while (rounds < MAX_ROUNDS && !mma_done) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" :: "r"(base + off[j]), "r"(v + j), "r"(v ^ rounds), "r"(v), "r"(v + rounds) : "memory");
+                if (p.fence & 1) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                ++rounds;
+            }
+        } else {
+            uint4 cur, cur2;
+            load2(0, cur, cur2);
+            while (rounds < MAX_ROUNDS && !mma_done) {
+                uint4 a = cur, b = cur2;
+                if (p.fence & 4) load2(rounds + 1, cur, cur2);
+                else { a.x += rounds; b.y ^= rounds; }
+                expand_store(a, b);
+                ++rounds;
+            }
         }
         if (r == 0) p.rounds[blockIdx.x] = (unsigned long long)rounds;
     }
@@ -115,12 +173,25 @@ int main()
     long long* hc = (long long*)malloc(sms * 8);
     unsigned long long* hr = (unsigned long long*)malloc(sms * 8);
     const int mma_count = 2048;
-    for (int fence = 0; fence < 2; ++fence)
-        for (int st : {0, 320, 640, 960})
+    uint4* gsrc; CK(cudaMalloc(&gsrc, (size_t)sms * 1024 * 64 * 16)); CK(cudaMemset(gsrc, 0x5a, (size_t)sms * 1024 * 64 * 16));
+    struct Mode { int bits; const char* name; };
+    const Mode modes[] = {{0, "stores"}, {1, "stores + fence"}, {3, "expansion + fence, no loads"},
+                          {7, "2 x 16-byte loads, 1 round ahead"}, {7 + 32, "1 x 32-byte load, 1 round ahead"},
+                          {7 + 16, "2 x 16-byte loads, 2 rounds ahead"}, {7 + 16 + 32, "1 x 32-byte load, 2 rounds ahead"},
+                          {7 + 64, "2 x 16-byte loads, 4 rounds ahead"}, {7 + 64 + 32, "1 x 32-byte load, 4 rounds ahead"}};
+    {
+        P p{gsrc, mma_count, 0, 0, clk, rounds, err};
+        for (int rep = 0; rep < 2; ++rep) { mma_with_stores<<<sms, 32, smem>>>(p); CK(cudaDeviceSynchronize()); }
+        CK(cudaMemcpy(hc, clk, sms * 8, cudaMemcpyDeviceToHost));
+        double c = 0;
+        for (int i = 0; i < sms; ++i) c += (double)hc[i];
+        printf("MMAs N 192 alone: %6.1f clocks per MMA\n", c / sms / mma_count);
+    }
+    for (const Mode& mode : modes)
+        for (int st : {320, 640, 960})
             for (int with_mma = 0; with_mma < 2; ++with_mma) {
-                if (!with_mma && st == 0) continue;
-                if (fence && st == 0) continue;
-                P p{with_mma ? mma_count : 0, st, fence, clk, rounds, err};
+                const int fence = mode.bits;
+                P p{gsrc, with_mma ? mma_count : 0, st, fence, clk, rounds, err};
                 CK(cudaMemset(rounds, 0, sms * 8));
                 for (int rep = 0; rep < 2; ++rep) { mma_with_stores<<<sms, 32 + (st > 0 ? st : 0), smem>>>(p); CK(cudaDeviceSynchronize()); }
                 CK(cudaMemcpy(hc, clk, sms * 8, cudaMemcpyDeviceToHost));
@@ -129,8 +200,8 @@ int main()
                 double c = 0, r = 0;
                 for (int i = 0; i < sms; ++i) { c += (double)hc[i]; r += (double)hr[i]; }
                 c /= sms; r /= sms;
-                printf("%-14s %3d storing threads%s: ", with_mma ? "MMAs N 192 +" : "no MMAs,", st, fence ? " (+ proxy fence per round)" : "");
-                if (with_mma) printf("%6.1f clocks per MMA (alone: 96.6 ideal); ", c / mma_count);
+                printf("%-36s %3d threads, %-13s ", mode.name, st, with_mma ? "beside MMAs:" : "no MMAs:");
+                if (with_mma) printf("%6.1f clocks per MMA; ", c / mma_count);
                 if (st > 0) printf("stores %6.1f bytes per clock per SM", r * st * 128.0 / c);
                 printf("%s\n", e ? "  (a wait ran out)" : "");
             }
