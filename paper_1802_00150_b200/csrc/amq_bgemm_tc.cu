@@ -90,6 +90,12 @@ struct TcParams {
     int pad;        // bit positions per row that are zero in both operands (they add +1 each to every dot product)
 };
 
+// Row stride (floats) of the epilogue's staging array y[plane-row][entry].  The plain product stores and reads it in
+// 128-bit pieces (four entries at a time: the epilogue's shared-memory instructions queue behind the expansion's in the
+// load/store unit, so their number counts), which wants a stride of 4 (mod 8) words for conflict-free quarter-warps; the cells
+// read it entry by entry with unit-strided rows and keep the odd stride.
+__host__ __device__ __forceinline__ int staging_stride(int TB, int epilogue) { return epilogue == EPI_Y ? TB + 4 : TB + 1; }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
@@ -378,7 +384,7 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
                                                       const float* sBcorr, float* Yt)
 {
     const GemmArgs& a = p.a;
-    const int k_w = a.k_w, n_mma = p.n_mma, ldy = p.TB + 1;
+    const int k_w = a.k_w, n_mma = p.n_mma, ldy = staging_stride(p.TB, a.epilogue);
     const int TMp = p.UT * p.gates * k_w;
     const int pr = quarter * 32 + lane;
     const int groups = p.TB >> 3;
@@ -407,7 +413,11 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
         }
         return;
     }
-    // loops without divisions: the per-item overhead is spread over only 8 * KA accumulators per thread
+    // loops without divisions: the per-item overhead is spread over only 8 * KA accumulators per thread.  This half of the
+    // epilogue is a chain of latencies, not of issue slots (about three instructions per accumulator); reading two items
+    // from tensor memory before folding the first was measured and lost (registers: the kernel's 1024-thread bound leaves
+    // 64, the second item spilled: C5 product 151 us against 120 us), and so was fetching the coefficients ahead of the
+    // tensor-memory wait (122 us)
     const bool fp4 = p.fp4 != 0;
     for (int mt = 0; mt < p.MT; ++mt)
     for (int seg = 0; seg < p.nseg; ++seg)
@@ -430,6 +440,7 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
             for (int q = 0; q < KA; ++q) b4[q] = reinterpret_cast<const float4*>(sBeta + (g * 8 + half * 4) * KA)[q];
             const float4 c4 = *reinterpret_cast<const float4*>(sBcorr + g * 8 + half * 4);
             const float corr4[4] = {c4.x, c4.y, c4.z, c4.w};
+            float y4[4];
 #pragma unroll
             for (int e4 = 0; e4 < 4; ++e4) {
                 float y = last ? corr4[e4] : 0.0f;
@@ -441,7 +452,13 @@ __device__ __forceinline__ void epilogue_tmem_to_smem(const TcParams& p, uint32_
                     const int col = (half * 4 + e4) * KA + j;
                     y += beta * acc_to_float(acc[col / 8][col % 8], fp4);
                 }
-                yrow[half * 4 + e4] = alpha * y;
+                y4[e4] = alpha * y;
+            }
+            if (a.epilogue == EPI_Y) {
+                *reinterpret_cast<float4*>(yrow + half * 4) = make_float4(y4[0], y4[1], y4[2], y4[3]);
+            } else {
+#pragma unroll
+                for (int e4 = 0; e4 < 4; ++e4) yrow[half * 4 + e4] = y4[e4];
             }
         }
     }
@@ -452,7 +469,7 @@ __device__ __forceinline__ void epilogue_smem_to_global(const TcParams& p, const
 {
     // thread -> (row or unit, every `bstep`-th batch entry): one division per thread, none per output
     const GemmArgs& a = p.a;
-    const int k_w = a.k_w, TB = p.TB, MT = p.MT, ldy = p.TB + 1;
+    const int k_w = a.k_w, TB = p.TB, MT = p.MT, ldy = staging_stride(p.TB, a.epilogue);
     const int TM = p.UT * p.gates;
     const int per_tile = (a.epilogue == EPI_Y) ? TM : p.UT;         // rows (plain) or units (cells) of an M tile
     const int items = MT * per_tile;
@@ -469,25 +486,17 @@ __device__ __forceinline__ void epilogue_smem_to_global(const TcParams& p, const
             const float bias = a.bias ? __ldg(a.bias + row) : 0.0f;
             const float* y0 = Yt + ((size_t)(mt * p.nseg) * TILE_M + li * k_w) * ldy;
             const int bend = (a.batch - b0 < TB) ? a.batch - b0 : TB;
-            int bb = bsub;
+            // four consecutive entries per item: one 128-bit load per plane, four stores (rows of y are entries)
             float* out = a.y + (size_t)b0 * a.ldy + row;
-            for (; bb + 7 * bstep < bend; bb += 8 * bstep) {       // eight entries in flight, planes unrolled
-                float s[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float* yq = y0 + bb + q * bstep;
-                    s[q] = bias + yq[0];
-                    if (k_w > 1) s[q] += yq[ldy];
-                    if (k_w > 2) s[q] += yq[2 * ldy];
-                    if (k_w > 3) s[q] += yq[3 * ldy];
-                }
-#pragma unroll
-                for (int q = 0; q < 8; ++q) out[(size_t)(bb + q * bstep) * a.ldy] = s[q];
-            }
-            for (; bb < bend; bb += bstep) {
-                float s = bias;
-                for (int i = 0; i < k_w; ++i) s += y0[i * ldy + bb];
-                a.y[(size_t)(b0 + bb) * a.ldy + row] = s;
+            for (int b4 = 4 * bsub; b4 < bend; b4 += 4 * bstep) {
+                float4 s = *reinterpret_cast<const float4*>(y0 + b4);
+                if (k_w > 1) { const float4 v = *reinterpret_cast<const float4*>(y0 + ldy + b4); s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+                if (k_w > 2) { const float4 v = *reinterpret_cast<const float4*>(y0 + 2 * ldy + b4); s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+                if (k_w > 3) { const float4 v = *reinterpret_cast<const float4*>(y0 + 3 * ldy + b4); s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+                out[(size_t)b4 * a.ldy] = bias + s.x;
+                if (b4 + 1 < bend) out[(size_t)(b4 + 1) * a.ldy] = bias + s.y;
+                if (b4 + 2 < bend) out[(size_t)(b4 + 2) * a.ldy] = bias + s.z;
+                if (b4 + 3 < bend) out[(size_t)(b4 + 3) * a.ldy] = bias + s.w;
             }
         } else if (a.epilogue == EPI_LSTM) {
             const int H = a.H, u = u0 + item;
@@ -788,7 +797,7 @@ bgemm_tc_kernel(TcParams p)
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
     // ---- epilogue: tensor memory -> partial products in shared memory (reusing the stage buffers) -> results ----
-    float* Yt = reinterpret_cast<float*>(smem_raw);                 // [MT][nseg][128][TB + 1]
+    float* Yt = reinterpret_cast<float*>(smem_raw);                 // [MT][nseg][128][staging_stride]
     const int epi_slots = mma_warp >> 2;                            // whole groups of four warps among the expanders
     if (warp < 4 * epi_slots)
         epilogue_tmem_to_smem<KA>(p, tmem_base, u0, b0, warp & 3, lane, warp >> 2, epi_slots, sAlpha, sBeta, sBcorr, Yt);
@@ -830,7 +839,7 @@ bgemm_tc_persistent_kernel(TcParams p)
     const int ntiles = p.ntiles, MG = p.mgroups, tile_step = (int)gridDim.x;
 
     unsigned char* stage_base = smem_raw;
-    float* Yt = reinterpret_cast<float*>(smem_raw + (size_t)S * stage_bytes);               // [MT][nseg][128][TB + 1]
+    float* Yt = reinterpret_cast<float*>(smem_raw + (size_t)S * stage_bytes);               // [MT][nseg][128][staging_stride]
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)S * stage_bytes + p.yt_bytes);   // [S]
     uint64_t* empty_bar = full_bar + MAX_STAGES;                                            // [S]
     uint64_t* tfull_bar = empty_bar + MAX_STAGES;                                           // [2] accumulator buffer complete
@@ -1146,7 +1155,7 @@ bool plan_persistent(const TcParams& base, int mtiles, int btiles, TcPlan* out)
     while (cols < p.nbuf * acc_cols + (p.fp4 ? 16 : 0)) cols <<= 1;
     p.tmem_cols = cols;
     const size_t stage = (size_t)128 * (TILE_M + p.n_mma);
-    p.yt_bytes = (int)(((size_t)p.nseg * TILE_M * (p.TB + 1) * 4 + 15) / 16 * 16);
+    p.yt_bytes = (int)(((size_t)p.nseg * TILE_M * staging_stride(p.TB, p.a.epilogue) * 4 + 15) / 16 * 16);
     const size_t fixed = (size_t)p.yt_bytes + (2 * MAX_STAGES + 4) * 8 + 16 + (2 * TILE_M + 256 + 128) * 4;
     int S = (int)((225 * 1024 - fixed) / stage);
     if (S > MAX_STAGES) S = MAX_STAGES;
@@ -1212,7 +1221,7 @@ bool plan(const GemmArgs& a, TcPlan* out)
     if (cols > 512) return false;
     p.tmem_cols = cols;
     const size_t stage = (size_t)128 * (p.MT * TILE_M + p.n_mma);
-    const size_t epi = (size_t)p.MT * p.nseg * TILE_M * (p.TB + 1) * 4;
+    const size_t epi = (size_t)p.MT * p.nseg * TILE_M * staging_stride(p.TB, a.epilogue) * 4;
     int S = (int)((220 * 1024) / stage);
     if (S > MAX_STAGES) S = MAX_STAGES;
     if (S < 2) return false;
