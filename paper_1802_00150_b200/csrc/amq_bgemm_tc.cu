@@ -88,6 +88,11 @@ struct TcParams {
     int sf_col;     // first tensor-memory column of the scale factors (all bytes 0x7F = 2^0)
     int steps;      // pipeline steps per tile: chunks of 128 bit positions, or pairs of them
     int pad;        // bit positions per row that are zero in both operands (they add +1 each to every dot product)
+    // persistent form, 4-bit operands: the weight operand of a pipeline step expanded into tensor memory (32 columns per
+    // stage, thread = plane-row = lane) instead of shared memory: its stores and the MMA's reads of it leave the
+    // load/store unit and the shared-memory port to the activation operand
+    int a_tmem;
+    int a_col;      // first tensor-memory column of the weight-operand stages
 };
 
 // Row stride (floats) of the epilogue's staging array y[plane-row][entry].  The plain product stores and reads it in
@@ -336,6 +341,54 @@ __device__ __forceinline__ void mma_mxf4_stage(uint32_t d_tmem, uint32_t a_lo, u
         "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %4, [%6], [%6], q;\n\t"
         "}"
         :: "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc_first), "r"(sf_tmem) : "memory");
+}
+
+// The same with the weight operand in tensor memory (lanes 0..127, 8 columns = 64 nibbles per MMA).
+__device__ __forceinline__ void mma_mxf4_stage_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                                  uint32_t acc_first, uint32_t sf_tmem)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .b64 db;\n\t"
+        ".reg .b32 al, bl;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "setp.eq.b32 q, %5, %5;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], [%1], db, %4, [%6], [%6], p;\n\t"
+        "add.u32 al, %1, 8;\n\t"
+        "add.u32 bl, %2, 2;\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], [al], db, %4, [%6], [%6], q;\n\t"
+        "add.u32 al, %1, 16;\n\t"
+        "add.u32 bl, %2, 4;\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], [al], db, %4, [%6], [%6], q;\n\t"
+        "add.u32 al, %1, 24;\n\t"
+        "add.u32 bl, %2, 6;\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], [al], db, %4, [%6], [%6], q;\n\t"
+        "}"
+        :: "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(acc_first), "r"(sf_tmem) : "memory");
+}
+
+// 4-bit form, weight operand in tensor memory: one 128-bit chunk of a packed row -> 16 columns of the thread's lane, in
+// the word order of the shared-memory row (word 4 q + s keeps bits s, s + 4, .. of packed word q).  Warp-collective.
+__device__ __forceinline__ void expand_chunk_fp4_tmem(uint32_t taddr, const uint4& v)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t y[16];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        y[4 * q + 0] = ((w[q] << 3) & 0x88888888u) | 0x22222222u;
+        y[4 * q + 1] = ((w[q] << 2) & 0x88888888u) | 0x22222222u;
+        y[4 * q + 2] = ((w[q] << 1) & 0x88888888u) | 0x22222222u;
+        y[4 * q + 3] = (w[q] & 0x88888888u) | 0x22222222u;
+    }
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        :: "r"(taddr), "r"(y[0]), "r"(y[1]), "r"(y[2]), "r"(y[3]), "r"(y[4]), "r"(y[5]), "r"(y[6]), "r"(y[7]),
+           "r"(y[8]), "r"(y[9]), "r"(y[10]), "r"(y[11]), "r"(y[12]), "r"(y[13]), "r"(y[14]), "r"(y[15]) : "memory");
 }
 
 // Scale factors of the 4-bit form: 16 tensor-memory columns, every byte 0x7F (2^0 in E8M0), written by four warps (one per
@@ -828,7 +881,8 @@ bgemm_tc_persistent_kernel(TcParams p)
     const int MT = p.MT, S = p.nstages, G = p.groups, EXP = p.expanders;
     const int mma_warp = (G * EXP) >> 5, epi_warp0 = mma_warp + 1, EW = p.epi_warps;
     const int n_mma = p.n_mma;
-    const int a_stage_bytes = MT * TILE_M * 128;
+    const bool a_tmem = FP4 && p.a_tmem != 0;       // weight operand in tensor memory: the stages hold the activation rows only
+    const int a_stage_bytes = a_tmem ? 0 : MT * TILE_M * 128;
     const int stage_bytes = a_stage_bytes + n_mma * 128;
     const int acc_cols = MT * p.nseg * n_mma;       // columns of one accumulator buffer
     const int CH = p.wpr >> 2;                      // 128-bit chunks along K
@@ -944,15 +998,24 @@ bgemm_tc_persistent_kernel(TcParams p)
             cur = nxt; cur2 = nxt2;
             pf_load(nxt, nxt2);
             if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity, failed)) { *failed = 1; break; }
-            if (writes) {
-                if (fp4) {
-                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off, v);
-                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off + 4, v2);
-                } else {
-                    expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, v, mul, m_sign, m_half);
+            if (a_tmem && is_a) {
+                // whole warps of weight rows: lane = plane-row mod 32, lane quarter = warp (the tile's 128 rows are warps 0..3)
+                const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(p.a_col + buf * 32);
+                expand_chunk_fp4_tmem(taddr, v);
+                expand_chunk_fp4_tmem(taddr + 16, v2);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            } else {
+                if (writes) {
+                    if (fp4) {
+                        expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off, v);
+                        expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off + 4, v2);
+                    } else {
+                        expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, v, mul, m_sign, m_half);
+                    }
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
             buf += G;
             if (buf >= S) { buf -= S; empty_parity ^= 1u; }
@@ -985,7 +1048,10 @@ bgemm_tc_persistent_kernel(TcParams p)
                         const int seg = word0 >= split_word ? 1 : 0;
                         const uint32_t acc_first = (word0 != 0 && word0 != split_word) ? 1u : 0u;
                         const uint32_t hi = (uint32_t)(desc_base >> 32);
-                        if (fp4) {
+                        if (a_tmem) {
+                            mma_mxf4_stage_ta(acc + seg * n_mma, tmem_base + (uint32_t)(p.a_col + buf * 32), (uint32_t)bdesc0, hi, idesc,
+                                              acc_first, sf_tmem);
+                        } else if (fp4) {
                             mma_mxf4_stage(acc + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first, sf_tmem);
                             if (MT == 2)
                                 mma_mxf4_stage(acc + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi,
@@ -1151,16 +1217,22 @@ bool plan_persistent(const TcParams& base, int mtiles, int btiles, TcPlan* out)
     p.sf_col = p.nbuf * acc_cols;
     p.steps = p.fp4 ? (CH + 1) / 2 : CH;
     p.pad = p.wpr * 32 - p.a.n + ((p.fp4 && (CH & 1)) ? 128 : 0);
-    int cols = 32;
-    while (cols < p.nbuf * acc_cols + (p.fp4 ? 16 : 0)) cols <<= 1;
-    p.tmem_cols = cols;
-    const size_t stage = (size_t)128 * (TILE_M + p.n_mma);
+    // the weight operand of the 4-bit form goes to tensor memory when at least three stages of 32 columns fit beside the
+    // accumulators and the scale factors
+    const int a_stages = p.fp4 ? (512 - (p.nbuf * acc_cols + 16)) / 32 : 0;
+    p.a_tmem = a_stages >= 3 ? 1 : 0;
+    p.a_col = p.sf_col + 16;
+    const size_t stage = (size_t)128 * ((p.a_tmem ? 0 : TILE_M) + p.n_mma);
     p.yt_bytes = (int)(((size_t)p.nseg * TILE_M * staging_stride(p.TB, p.a.epilogue) * 4 + 15) / 16 * 16);
     const size_t fixed = (size_t)p.yt_bytes + (2 * MAX_STAGES + 4) * 8 + 16 + (2 * TILE_M + 256 + 128) * 4;
     int S = (int)((225 * 1024 - fixed) / stage);
     if (S > MAX_STAGES) S = MAX_STAGES;
+    if (p.a_tmem && S > a_stages) S = a_stages;
     if (S < 2) return false;
     p.nstages = S;
+    int cols = 32;
+    while (cols < p.nbuf * acc_cols + (p.fp4 ? 16 : 0) + (p.a_tmem ? 32 * S : 0)) cols <<= 1;
+    p.tmem_cols = cols;
     p.expanders = (TILE_M + p.n_mma + 31) / 32 * 32;
     // one expander group; eight epilogue warps, or up to sixteen where the MMAs of the next tile have to wait for the
     // epilogue (one accumulator buffer; measured: C4 timestep 53.7 -> 50.3 us, nothing gained with two buffers)
