@@ -614,7 +614,8 @@ bgemm_tc_kernel(TcParams p)
     const int EXP = p.expanders;                    // operand rows rounded up to whole warps
     const int mma_warp = (G * EXP) >> 5, nthreads = G * EXP + 32;
     const int n_mma = p.n_mma;
-    const int a_stage_bytes = MT * TILE_M * 128;    // 128 bytes of K per row and stage
+    const bool a_tmem = FP4 && p.a_tmem != 0;       // weight operand in tensor memory (one M tile): the stages hold the activation rows
+    const int a_stage_bytes = a_tmem ? 0 : MT * TILE_M * 128;       // 128 bytes of K per row and stage
     const int stage_bytes = a_stage_bytes + n_mma * 128;
     const int u0 = blockIdx.x * p.UT * MT, b0 = blockIdx.y * p.TB;
 
@@ -660,7 +661,9 @@ bgemm_tc_kernel(TcParams p)
     uint4 cur = zero, cur2 = zero, nxt = zero, nxt2 = zero;
     if (expander) {
         if (weight_row) {
-            const int mt = r_all >> 7, r = r_all & (TILE_M - 1);
+            // with the operand in tensor memory a warp can only write the lane quarter (warp mod 4): the four weight warps
+            // of a group (consecutive warps) take the row blocks in that order
+            const int mt = r_all >> 7, r = a_tmem ? ((warp & 3) << 5) | lane : r_all & (TILE_M - 1);
             size_t prow = 0;                                        // plane-row index in Wcodes / Walpha
             if (r < TMp) {
                 const int l = div_small(r, k_w), i = r - l * k_w;
@@ -673,7 +676,7 @@ bgemm_tc_kernel(TcParams p)
             }
             dst0 = smem_u32(stage_base) + r_all * 128;
             if (grp == 0) {
-                coef_dst = sAlpha + r_all;
+                coef_dst = sAlpha + mt * TILE_M + r;
                 if (src && a.epilogue != EPI_DOTS) coef_src = a.Walpha + prow;
             }
         } else {
@@ -748,15 +751,23 @@ bgemm_tc_kernel(TcParams p)
         // one pipeline step: the MMAs that read this buffer one lap ago must have completed; expand; hand over
         auto step = [&](const uint4& lo, const uint4& hi) {
             if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; go_on = false; return; }
-            if (writes) {
-                if (fp4) {
-                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off, lo);
-                    expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off + 4, hi);
-                } else {
-                    expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, lo, mul, m_sign, m_half);
+            if (a_tmem && weight_row) {
+                const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(p.a_col + buf * 32);
+                expand_chunk_fp4_tmem(taddr, lo);
+                expand_chunk_fp4_tmem(taddr + 16, hi);
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            } else {
+                if (writes) {
+                    if (fp4) {
+                        expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off, lo);
+                        expand_chunk_fp4(dst0 + (uint32_t)(buf * stage_bytes), off + 4, hi);
+                    } else {
+                        expand_chunk(dst0 + (uint32_t)(buf * stage_bytes), off, lo, mul, m_sign, m_half);
+                    }
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // generic-proxy stores -> async proxy
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(&full_bar[buf])) : "memory");
         };
         for (int q = grp; q < PAIRS && go_on; q += G) {
@@ -805,7 +816,10 @@ bgemm_tc_kernel(TcParams p)
                 const int seg = word0 >= split_word ? 1 : 0;
                 const uint32_t acc_first = (word0 != 0 && word0 != split_word) ? 1u : 0u;
                 const uint32_t hi = (uint32_t)(desc_base >> 32);
-                if (fp4) {
+                if (a_tmem) {
+                    mma_mxf4_stage_ta(tmem_base + seg * n_mma, tmem_base + (uint32_t)(p.a_col + buf * 32), (uint32_t)bdesc0, hi, idesc,
+                                      acc_first, sf_tmem);
+                } else if (fp4) {
                     mma_mxf4_stage(tmem_base + seg * n_mma, (uint32_t)adesc0, (uint32_t)bdesc0, hi, idesc, acc_first, sf_tmem);
                     if (MT == 2)
                         mma_mxf4_stage(tmem_base + (p.nseg + seg) * n_mma, (uint32_t)adesc0 + (TILE_M * 128 >> 4), (uint32_t)bdesc0, hi,
@@ -1288,17 +1302,23 @@ bool plan(const GemmArgs& a, TcPlan* out)
     p.sf_col = acc_cols;
     p.steps = p.fp4 ? (CH + 1) / 2 : CH;
     p.pad = p.wpr * 32 - a.n + ((p.fp4 && (CH & 1)) ? 128 : 0);
-    int cols = 32;
-    while (cols < acc_cols + (p.fp4 ? 16 : 0)) cols <<= 1;
-    if (cols > 512) return false;
-    p.tmem_cols = cols;
-    const size_t stage = (size_t)128 * (p.MT * TILE_M + p.n_mma);
+    // with one M tile per CTA the weight operand of the 4-bit form goes to tensor memory when at least three stages of 32
+    // columns fit beside the accumulators and the scale factors (and the epilogue's staging array still fits the stages)
+    const int a_stages = (p.fp4 && p.MT == 1) ? (512 - (acc_cols + 16)) / 32 : 0;
     const size_t epi = (size_t)p.MT * p.nseg * TILE_M * staging_stride(p.TB, a.epilogue) * 4;
+    p.a_tmem = (a_stages >= 3 && epi <= (size_t)(a_stages < MAX_STAGES ? a_stages : MAX_STAGES) * 128 * p.n_mma) ? 1 : 0;
+    p.a_col = p.sf_col + 16;
+    const size_t stage = (size_t)128 * ((p.a_tmem ? 0 : p.MT * TILE_M) + p.n_mma);
     int S = (int)((220 * 1024) / stage);
     if (S > MAX_STAGES) S = MAX_STAGES;
+    if (p.a_tmem && S > a_stages) S = a_stages;
     if (S < 2) return false;
     if (epi > S * stage) return false;
     p.nstages = S;
+    int cols = 32;
+    while (cols < acc_cols + (p.fp4 ? 16 : 0) + (p.a_tmem ? 32 * S : 0)) cols <<= 1;
+    if (cols > 512) return false;
+    p.tmem_cols = cols;
     p.expanders = (p.MT * TILE_M + p.n_mma + 31) / 32 * 32;
     p.groups = (2 * p.expanders + 32 <= MAX_THREADS) ? 2 : 1;
     out->p = p;
