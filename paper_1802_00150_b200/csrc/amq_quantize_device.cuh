@@ -258,9 +258,12 @@ __device__ __forceinline__ void level_table(const float (&alpha)[K], int lane, f
     __syncwarp();
 #pragma unroll
     for (int p = 0; p < M - 1; ++p) thr[p] = (sc_level[p] + sc_level[p + 1]) * 0.5f;
+    // bit p of plane[i] = sign of plane i in the code at sorted position p: lane p holds that code, one ballot per plane
+    // (the same masks as planes_from_table builds from the packed table, in a tenth of the instructions)
+    const int code = lane < M ? sc_code[lane] : 0;
 #pragma unroll
-    for (int p = 0; p < M; ++p) table |= (unsigned long long)sc_code[p] << (4 * p);
-    planes_from_table<K>(table, plane);
+    for (int i = 0; i < K; ++i) plane[i] = __ballot_sync(0xffffffffu, ((code >> (K - 1 - i)) & 1) != 0);
+    (void)table;
 }
 
 // Algorithm 1 for one element: index of the leaf (sorted level) the descent over the midpoints reaches.
