@@ -35,6 +35,15 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_write.sum), keyed by workload; the summaries are under profiles/.  None = not captured for the
 # kernel as it stands.
 NCU_TRAFFIC_BYTES = {"lstm1024_b1": 2422016 + 51968}    # rnn_persistent_kernel, profiles/rnn_persistent_kernel_lstm1024_b1.txt
+# the batched workloads time a chain of kernels; for their dominant kernel (the tensor-core product) the cold-cache ncu
+# captures under profiles/ give these DRAM bytes per launch (inside a sequence the packed weights stay in L2)
+NCU_TRAFFIC_DOMINANT_KERNEL = {
+    "lstm1024_b64": {"kernel": "bgemm_tc_kernel", "bytes": 3586816, "summary": "profiles/bgemm_tc_kernel_lstm1024_b64.txt"},
+    "gru2048_b256": {"kernel": "bgemm_tc_persistent_kernel", "bytes": 8923136,
+                     "summary": "profiles/bgemm_tc_persistent_kernel_gru2048_b256.txt"},
+    "proj32768_b512": {"kernel": "bgemm_tc_persistent_kernel", "bytes": 13188352 + 10061568,
+                       "summary": "profiles/bgemm_tc_persistent_kernel_proj32768_b512.txt"},
+}
 # the same for the cold matrix-vector kernel on 131072 x 8192 at 2/2 bits (profiles/bgemv_kernel_131072x8192_k2k2.txt)
 NCU_TRAFFIC_GEMV_COLD_BYTES = 269500000
 
@@ -414,6 +423,8 @@ def run_ours(args, wl):
                          "traffic": NCU_TRAFFIC_BYTES.get(wl.name)},
             "us_per_timestep": 1e3 * step_ms / max(wl.steps, 1) if wl.cell != "proj" else None,
         }
+        if wl.name in NCU_TRAFFIC_DOMINANT_KERNEL:
+            line["roofline"]["traffic_dominant_kernel"] = NCU_TRAFFIC_DOMINANT_KERNEL[wl.name]
         if not args.no_extras and world == 1:
             line["gemv_cold"] = cold_gemv(amq, torch, dev, flush, peak, peak_kind)
             # the second half of the metric (binary matrix-vector product against the HBM peak) beside the first
