@@ -750,7 +750,10 @@ bgemm_tc_kernel(TcParams p)
         bool go_on = true;
         // one pipeline step: the MMAs that read this buffer one lap ago must have completed; expand; hand over
         auto step = [&](const uint4& lo, const uint4& hi) {
-            if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity)) { *failed = 1; go_on = false; return; }
+            bool free_now = mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity);
+            // (the tensor-memory stores below are warp-collective: a weight warp gives up as a whole or not at all)
+            if (a_tmem && weight_row) free_now = __all_sync(0xffffffffu, free_now);
+            if (!free_now) { *failed = 1; go_on = false; return; }
             if (a_tmem && weight_row) {
                 const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(p.a_col + buf * 32);
                 expand_chunk_fp4_tmem(taddr, lo);
@@ -1011,7 +1014,10 @@ bgemm_tc_persistent_kernel(TcParams p)
             const uint4 v = cur, v2 = cur2;
             cur = nxt; cur2 = nxt2;
             pf_load(nxt, nxt2);
-            if (!mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity, failed)) { *failed = 1; break; }
+            bool free_now = mbar_wait_relaxed(smem_u32(&empty_bar[buf]), empty_parity, failed);
+            // (the tensor-memory stores below are warp-collective: a weight warp gives up as a whole or not at all)
+            if (a_tmem && is_a) free_now = __all_sync(0xffffffffu, free_now);
+            if (!free_now) { *failed = 1; break; }
             if (a_tmem && is_a) {
                 // whole warps of weight rows: lane = plane-row mod 32, lane quarter = warp (the tile's 128 rows are warps 0..3)
                 const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(p.a_col + buf * 32);
