@@ -174,6 +174,30 @@ GEMM_CASES = [
 ]
 
 
+def offset_by_16_bytes(c):
+    """The packed planes on the device, starting 16 bytes past a 32-byte boundary."""
+    flat = np.ascontiguousarray(c).view(np.int32).reshape(-1)
+    buf = torch.zeros(flat.size + 12, dtype=torch.int32, device="cuda")
+    start = ((-(buf.data_ptr() // 4)) % 8 + 4) % 8          # first word whose address is 16 (mod 32)
+    view = buf[start:start + flat.size]
+    view.copy_(torch.from_numpy(flat).cuda())
+    assert view.data_ptr() % 32 == 16
+    return view.view(c.shape)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("m,n,kw,ka,batch", [(257, 512, 1, 4, 17), (130, 2048, 3, 3, 64), (2500, 300, 4, 4, 70), (6144, 256, 2, 3, 250)])
+def test_dots_bit_exact_with_planes_on_16_byte_boundaries(amq, m, n, kw, ka, batch):
+    # the tensor-core kernels fetch 32 bytes of a row at a time where the row is 32-byte aligned and fall back to
+    # 16-byte loads where it is not: here no row is (even strides), or every other one (n = 300)
+    W = synth.normal((m, n), 0.03, 70 + m, 1).astype(np.float64)
+    X = synth.uniform((batch, n), -1, 1, 70 + m, 2).astype(np.float64)
+    Wc, _ = oracle.quantize_rows(W, kw, 2)
+    Xc, _ = oracle.quantize_rows(X, ka, 2)
+    D = amq.binary_dots(offset_by_16_bytes(Wc), offset_by_16_bytes(Xc), n).cpu().numpy()
+    assert np.array_equal(D, oracle.binary_dots(Wc, Xc, n))
+
+
 @pytest.mark.parametrize("m,n,kw,ka,batch", GEMM_CASES)
 def test_dots_bit_exact_and_product_within_tolerance(amq, m, n, kw, ka, batch):
     W = synth.normal((m, n), 0.03, 20 + m, 1).astype(np.float64)
