@@ -332,6 +332,9 @@ AMQ_API amq_status amq_lm_greedy_decode(const uint32_t* We_codes, const float* W
  * (pinned memory makes the copies asynchronous) into `staging`, the sequence runs, and h_last / c_last
  * (and h_seq when not NULL) are copied back to host memory; the call returns after the stream has
  * drained.  Weights, bias, workspace and staging (amq_cell_host_staging_bytes) stay DEVICE pointers.
+ * Inputs of 4 MiB and more of a batched sequence are copied in up to eight chunks of timesteps on a stream that
+ * the call creates and destroys, so that the copy of later timesteps runs beside the kernels of earlier ones;
+ * the results do not depend on it.
  */
 AMQ_API amq_status amq_lstm_sequence_host(const uint32_t* Wcodes, const float* Walpha, const float* bias,
                                   int I, int H, int k_w,

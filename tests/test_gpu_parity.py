@@ -370,6 +370,28 @@ def test_sequence_host_variant(amq):
     assert torch.equal(gh, g2.cpu())
 
 
+def test_sequence_host_variant_with_inputs_copied_in_chunks(amq):
+    # inputs of more than 4 MiB reach a batched chain in chunks of timesteps on a stream of their own, beside the kernels
+    # of the earlier timesteps: the results must be those of the device-resident call, bit for bit, run after run
+    I, H, batch, steps, ka = 1024, 96, 40, 29, 3
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    dWc, dWa = amq.quantize(torch.randn((4 * H, I + H), device="cuda", generator=g) * 0.05, 2, 2)
+    xs = torch.from_numpy(synth.normal((steps, batch, I), 1.0, 63, 1)).pin_memory()
+    assert xs.numel() * 4 >= 4 << 20
+    h0 = torch.from_numpy(synth.uniform((batch, H), -1, 1, 63, 2)).pin_memory()
+    c0 = torch.from_numpy(synth.uniform((batch, H), -1, 1, 63, 3)).pin_memory()
+    ws = amq.new_workspace(I, H, batch, ka)
+    st = amq.new_host_staging(I, H, batch, steps)
+    g_seq, g_last, g_c = amq.lstm_sequence(dWc, dWa, None, I, H, xs.cuda(), h0.cuda(), c0.cuda(), ka, 2, ws, want_h_seq=True)
+    for _ in range(3):
+        h_last, c_last = torch.zeros((batch, H)).pin_memory(), torch.zeros((batch, H)).pin_memory()
+        h_seq = torch.zeros((steps, batch, H)).pin_memory()
+        st.zero_()
+        amq.lstm_sequence_host(dWc, dWa, None, I, H, xs, h0, c0, ka, 2, ws, st, h_last, c_last, h_seq=h_seq)
+        assert torch.equal(h_seq, g_seq.cpu()) and torch.equal(h_last, g_last.cpu()) and torch.equal(c_last, g_c.cpu())
+    assert amq.workspace_status(ws) == 0 and amq.device_status() == 0
+
+
 def test_empty_batch_and_zero_steps(amq):
     I, H, ka = 32, 32, 2
     Wc, Wa, bias = cell_setup("lstm", I, H, 2, 70, 0.08)
