@@ -126,6 +126,11 @@ AMQ_API amq_status amq_binary_dots(const uint32_t* Wcodes, int m, int n, int k_w
  *   y[b][r] = sum_i sum_j Walpha[r][i] * xbeta[b][j] * D[b][r][i][j] + bias[r].
  * Walpha [m][k_w], xbeta [batch][k_a], bias [m] or NULL, y [batch][ldy] fp32 out, ldy >= m.
  * The integer partials are exact; the combination is fp32.
+ * Wcodes and xcodes must be 16-byte aligned (AMQ_ERR_ALIGNMENT otherwise).  From 16 vectors on the product runs on
+ * the tensor cores; its kernels fetch 32 bytes of a packed row at a time where the row starts on a 32-byte boundary
+ * (a 32-byte aligned base with an even number of 128-element chunks per row, as torch allocations give for
+ * n a multiple of 256) and fall back to 16-byte loads elsewhere: same results, about a fifth slower on large
+ * products.
  */
 AMQ_API amq_status amq_binary_gemm(const uint32_t* Wcodes, const float* Walpha, int m, int n, int k_w,
                            const uint32_t* xcodes, const float* xbeta, int batch, int k_a,
