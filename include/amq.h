@@ -82,7 +82,7 @@ AMQ_API size_t amq_codes_bytes(int rows, int n, int k);
  * with plane 0 the most significant code bit; a refit whose k x k system has a pivot below 1e-9 * n
  * (Gaussian elimination with partial pivoting, in double) is skipped and keeps the previous coefficients.
  * Sums over a row are accumulated in fp32 (per thread, then across threads in a fixed order, so results repeat
- * bit for bit); B^T B is exact integer arithmetic; the k x k solve is fp64 for k >= 3 and error-compensated fp32 for
+ * bit for bit); B^T B is exact integer arithmetic; the k x k solve is fp64 for k >= 3 (k = 3: adjugate of the exact integers) and error-compensated fp32 for
  * k = 2; levels, thresholds and comparisons are fp32.
  */
 AMQ_API amq_status amq_quantize(const float* x, int rows, int n, int ldx, int k, int T,

@@ -21,7 +21,7 @@
 //
 // Arithmetic: sums over the vector are fp32 (per thread, then a fixed butterfly over the warp, then the
 // per-warp partials in a fixed tree, so results are reproducible run to run); the Gram matrix B^T B is exact
-// integer arithmetic; the k x k solve is fp64 for k >= 3 and error-compensated fp32 for k = 2 (the products
+// integer arithmetic; the k x k solve is fp64 for k >= 3 (k = 3: through the exact integer adjugate) and error-compensated fp32 for k = 2 (the products
 // n c_i and g c_j are split exactly with fused multiply-adds, so cancellation costs nothing); levels,
 // midpoints and comparisons are fp32.
 //
@@ -112,7 +112,8 @@ __device__ __forceinline__ void group_totals(float (&f)[VF], int (&iv)[VI > 0 ? 
 
 // Least-squares solve of Eq. 5, G a = c with G = B^T B (G_ii = n, integer off-diagonals in gram[], row
 // major upper triangle).  Leaves `a` untouched and returns false when a pivot of Gaussian elimination with
-// partial pivoting falls below 1e-9 * n (reading for a singular system: skip the refit).
+// partial pivoting falls below 1e-9 * n (reading for a singular system: skip the refit).  k = 2 and k = 3 solve
+// through the exact integer adjugate (same rule, evaluated on exact quantities); k = 4 eliminates in fp64.
 template <int K>
 __device__ __forceinline__ bool solve_refit(const float (&c)[K], const int (&gram)[K > 1 ? K * (K - 1) / 2 : 1], int n,
                                             float (&a)[K])
@@ -136,6 +137,27 @@ __device__ __forceinline__ bool solve_refit(const float (&c)[K], const int (&gra
         const float t1 = fg * c[0], e1 = fmaf(fg, c[0], -t1);
         a[0] = (fmaf(fn, c[0], -t0) - e0) * rdet;
         a[1] = (fmaf(fn, c[1], -t1) - e1) * rdet;
+        return true;
+    }
+    if (K == 3) {
+        // Adjugate of the Gram matrix: its entries and the determinant are integers below 2^53, exact in fp64, so the only
+        // roundings are those of the three-term sums and of the division, and the dependent chain is a third of the
+        // elimination's (the solve is per-vector scalar work that every warp repeats; on the batched cells' on-line
+        // quantizer it was a visible part of a timestep).  The singularity rule is the elimination's, evaluated on the same
+        // exact quantities: its second pivot is max(|n^2 - g01^2|, |n g12 - g01 g02|) / n and its third
+        // |det| / (n x second pivot), whichever row the pivoting takes.
+        const double n_ = (double)n, g01 = (double)gram[0], g02 = (double)gram[1], g12 = (double)gram[2];
+        const double A00 = n_ * n_ - g12 * g12, A01 = g02 * g12 - g01 * n_, A02 = g01 * g12 - g02 * n_;
+        const double A11 = n_ * n_ - g02 * g02, A12 = g01 * g02 - g12 * n_, A22 = n_ * n_ - g01 * g01;
+        const double det = n_ * A00 + g01 * A01 + g02 * A02;
+        const double tiny = 1e-9 * n_;
+        const double pivot2n = fmax(fabs(A22), fabs(A12));          // n x the second pivot
+        if (!(pivot2n >= tiny * n_) || !(fabs(det) >= tiny * pivot2n)) return false;
+        const double rd = 1.0 / det;
+        const double c0 = (double)c[0], c1 = (double)c[1], c2 = (double)c[2];
+        a[0] = (float)((A00 * c0 + A01 * c1 + A02 * c2) * rd);
+        a[1] = (float)((A01 * c0 + A11 * c1 + A12 * c2) * rd);
+        a[2] = (float)((A02 * c0 + A12 * c1 + A22 * c2) * rd);
         return true;
     }
     double G[K][K + 1];
